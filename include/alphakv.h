@@ -1,0 +1,189 @@
+/*
+ * alphakv -- KV-cache compression event of the alpha retainer, CUDA (sm_100a).
+ *
+ * One *event* is one (sequence, layer, KV head). For every event the library
+ *   1. scores each cached token (alpha_score),
+ *   2. picks `budget` tokens with the greedy set-conditioned rule
+ *        Delta(i | S) = s_i - lambda * max(0, max_{j in S} cos(v_i, v_j))      (Eq. 2)
+ *        i_{t+1} = argmax_{i not in S_t} Delta(i | S_t),  i_1 = argmax s       (Eq. 3)
+ *      which at lambda = 0 is exactly top-k (Section 4.1, Algorithm 1)         (alpha_select),
+ *   3. moves the kept K/V rows to slots 0..budget-1 of the same buffer         (kv_compact),
+ * or does all three in one call (alpha_compress_event).
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C linkage; no C++/torch types. Every tensor pointer is DEVICE memory
+ *     owned by the caller and is not retained after the call. Scalars, the
+ *     layout and the options are HOST structs read during the call.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream). The return code reports host-side validation
+ *     and launch errors only; nothing is launched when it is not AKV_OK.
+ *   - No exceptions, aborts or exits. akv_last_error() gives a message for the
+ *     last failure on the calling thread.
+ *   - Tensors are addressed [B, L, H, N, d]: B sequences, L layers, H KV heads,
+ *     N slots per (sequence, layer, head), d head dimension (contiguous).
+ *     d must be a multiple of 8 and at most 256; row starts must be 16-byte
+ *     aligned (base pointers 16-byte aligned, strides multiples of 16 bytes).
+ *   - Per-event status words (device, int32 [B, L, H], optional):
+ *       0 ok; 1 a non-finite score was seen (such a token is never preferred);
+ *       2 fewer candidates than the budget (all are kept, n_kept < budget,
+ *         unused idx entries are -1); 3 an internal bounded wait gave up.
+ *   - Ties in any argmax go to the lower slot index.
+ */
+#ifndef ALPHAKV_H
+#define ALPHAKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct akv_handle akv_handle_t; /* opaque; owns only its own scratch workspace */
+
+typedef enum {
+    AKV_OK = 0,
+    AKV_ERR_INVALID_ARG = 1, /* null pointer, bad shape, negative lambda, ... */
+    AKV_ERR_UNSUPPORTED = 2, /* d, dtype or mode outside what is built */
+    AKV_ERR_BUDGET = 3,      /* budget < 1 or budget > N */
+    AKV_ERR_ALIGNMENT = 4,   /* pointer or stride breaks the 16-byte rule */
+    AKV_ERR_WORKSPACE = 5,   /* scratch could not be provided */
+    AKV_ERR_CUDA = 6         /* a CUDA runtime call failed (see akv_last_error) */
+} akv_status_t;
+
+typedef enum { AKV_F32 = 0, AKV_BF16 = 1 } akv_dtype_t;
+
+/* What V-space the cosine of Eq. 2 is taken in. PER_HEAD: the event's own V rows
+ * (Eq. 1 with the layer/head sums reduced to the one head; the variant Section 6
+ * names). FLAT: Eq. 1 literally, one signature per (sequence, slot) shared by all
+ * heads, produced by alpha_signature_flat. */
+typedef enum { AKV_SIG_PER_HEAD = 0, AKV_SIG_FLAT = 1 } akv_sig_mode_t;
+
+/* Layout of K and of V (both use the same one). Strides are in ELEMENTS.
+ * Dense (page_size == 0): row (b,l,h,n) starts at
+ *     b*stride_b + l*stride_l + h*stride_h + n*stride_n.
+ * Paged (page_size > 0, a power of two): slot n of sequence b lives in page
+ *     p = block_table[b*pages_per_seq + n/page_size] and row (b,l,h,n) starts at
+ *     l*stride_l + p*stride_page + h*stride_page_h + (n % page_size)*stride_page_n.
+ *   (stride_b, stride_h, stride_n are ignored.) N must be <= pages_per_seq*page_size.
+ */
+typedef struct {
+    int32_t B, L, H, N, d;
+    akv_dtype_t dtype;
+    int64_t stride_b, stride_l, stride_h, stride_n;
+    int32_t page_size;
+    const int32_t* block_table; /* device, int32 [B, pages_per_seq]; paged only */
+    int32_t pages_per_seq;
+    int64_t stride_page, stride_page_h, stride_page_n;
+} akv_layout_t;
+
+#define AKV_FLAG_FORCE_GREEDY 1u /* run the greedy loop even at lambda == 0 (testing aid) */
+#define AKV_FLAG_NO_PRUNE 2u     /* never shrink the candidate pool before the loop (testing aid) */
+
+typedef struct {
+    float lambda;          /* >= 0; 0 takes the top-k branch of Algorithm 1 */
+    float eps;             /* epsilon of Eq. 1: v = u / (||u||_2 + eps); default 1e-8 */
+    float rope_base;       /* RoPE base, default 10000 */
+    int32_t future_window; /* W >= 1 future query positions averaged by the score; default 1 */
+    akv_sig_mode_t sig_mode;
+    uint32_t flags;
+} akv_options_t;
+
+/* Fills *opt with the defaults named above (lambda = 0.5, the value the paper settles on). */
+void akv_default_options(akv_options_t* opt);
+
+/* Creates a handle bound to CUDA device `device`. The handle keeps a grow-only
+ * scratch buffer (cudaMalloc on first need, freed by akv_destroy). One handle
+ * must not be used from two host threads at once. */
+akv_status_t akv_create(akv_handle_t** out, int device);
+akv_status_t akv_destroy(akv_handle_t* h);
+/* Message for the most recent error on the calling thread; static storage. */
+const char* akv_last_error(void);
+const char* akv_status_string(akv_status_t s);
+/* Number of kernels this library has launched so far in this process. */
+uint64_t akv_launch_count(void);
+
+/*
+ * alpha_score -- per-token retention score s (Section 4.1: the scores "produced by
+ * the TriAttention 1d scorer"; the paper does not print the formula, the library
+ * uses: keys are stored pre-RoPE, coordinate f pairs with f + d/2,
+ *   s_i = (1/sqrt d) Re sum_f c_f z(q)_f conj(z(k_i)_f) exp(i (p_ref - p_i) theta_f),
+ *   theta_f = rope_base^(-2f/d), c_f = (1/W) sum_{w<W} exp(i w theta_f),
+ *   z(x)_f = x_f + i x_{f+d/2},
+ * the mean RoPE attention logit of the head's query statistic at positions
+ * p_ref..p_ref+W-1 against key i at p_i).
+ *   K       device, layout `lay`, read only.
+ *   pos     device int32, slot positions; element (b,l,h,n) at
+ *           b*pos_stride_b + l*pos_stride_l + h*pos_stride_h + n (a stride of 0
+ *           broadcasts). NULL: keys are already rotated, s_i = q . k_i / sqrt d.
+ *   n_cand  device int32 [B] valid slots per sequence, or NULL for N.
+ *   qstat   device fp32 [L, H, d] query statistic per KV head (for grouped-query
+ *           attention the caller averages its query heads; the score is linear in q).
+ *   p_ref   device int32 [B], or NULL for (largest position of the event) + 1.
+ *   scores  device fp32 [B, L, H, N] out; slots >= n_cand are left untouched.
+ *   status  device int32 [B, L, H] out or NULL.
+ */
+akv_status_t alpha_score(akv_handle_t* h, const akv_layout_t* lay, const void* K, const int32_t* pos,
+                         int64_t pos_stride_b, int64_t pos_stride_l, int64_t pos_stride_h,
+                         const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
+                         const akv_options_t* opt, float* scores, int32_t* status, void* stream);
+
+/*
+ * alpha_select -- Algorithm 1: greedy fill of the budget under Eq. 2 / Eq. 3, or
+ * top-k when lambda == 0. fp32 accumulation; cos(v_i, v_j) = <V_i, V_j> r_i r_j
+ * with r = 1 / (||V||_2 + eps) (Eq. 1's normalisation).
+ *   scores     device fp32 [B, L, H, N] in.
+ *   V          device, layout `lay`, read only (PER_HEAD mode); may be NULL in FLAT mode.
+ *   flat_sig   device fp32 [B, N, d], FLAT mode only (from alpha_signature_flat), else NULL.
+ *   budget     1 <= budget <= N (the paper's k).
+ *   idx_sorted device int32 [B, L, H, budget] out: sort(S), ascending slot index.
+ *   pick_order device int32 [B, L, H, budget] out or NULL: i_1, i_2, ... in pick order.
+ *   pick_gain  device fp32  [B, L, H, budget] out or NULL: Delta(i_t | S_{t-1}) at each pick.
+ *   n_kept     device int32 [B, L, H] out or NULL: min(budget, n_cand).
+ */
+akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, const float* scores, const void* V,
+                          const float* flat_sig, const int32_t* n_cand, int32_t budget,
+                          const akv_options_t* opt, int32_t* idx_sorted, int32_t* pick_order,
+                          float* pick_gain, int32_t* n_kept, int32_t* status, void* stream);
+
+/*
+ * alpha_signature_flat -- Eq. 1: u_i = (1/(L H)) sum_l sum_h V_i^(l,h), v_i = u_i / (||u_i||_2 + eps),
+ * one signature per (sequence, slot); slots must mean the same token in every head.
+ *   flat_sig  device fp32 [B, N, d] out (unit-normalised rows).
+ */
+akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+                                  const int32_t* n_cand, const akv_options_t* opt, float* flat_sig,
+                                  void* stream);
+
+/*
+ * kv_compact -- the retained rows become the new cache (Section 1; Section 4.1:
+ * "k <= n is the post-compression budget"): for r = 0..budget-1, row idx_sorted[r]
+ * of K, of V and of pos moves to slot r of the SAME buffer (bit copies). Entries
+ * idx_sorted[r] < 0 end the list. idx_sorted must be ascending and distinct (as
+ * alpha_select writes it); rows at slots >= the kept count are unspecified afterwards.
+ *   K, V  device, layout `lay`, rewritten in place (either may be NULL to skip it).
+ *   pos   device int32 with the strides above, rewritten in place, or NULL. When given,
+ *         its strides must address a distinct row per event (no broadcast).
+ */
+akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                        int64_t pos_stride_b, int64_t pos_stride_l, int64_t pos_stride_h,
+                        const int32_t* idx_sorted, int32_t budget, void* stream);
+
+/*
+ * alpha_compress_event -- score, select, order and compact in one call; K and V
+ * cross HBM once when an event's tiles fit on chip. Arguments as in the three
+ * calls above. K, V and pos are rewritten in place (pos may be NULL: already-rotated
+ * keys, nothing to carry). Outputs other than idx_sorted are optional (NULL skips).
+ *   scores  device fp32 [B, L, H, N] out or NULL.
+ */
+akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                  int64_t pos_stride_b, int64_t pos_stride_l, int64_t pos_stride_h,
+                                  const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
+                                  const float* flat_sig, int32_t budget, const akv_options_t* opt,
+                                  int32_t* idx_sorted, int32_t* pick_order, float* pick_gain,
+                                  float* scores, int32_t* n_kept, int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALPHAKV_H */

@@ -97,10 +97,14 @@ void orc_signature(const void* V, int dtype, int n, int d, double eps, double* s
     }
 }
 
-static int argmax_lowest(const double* a, int n) {
-    int best = 0;
-    for (int i = 1; i < n; ++i)
-        if (a[i] > a[best]) best = i;
+/* argmax over candidates not yet in S, ties to the lowest index; a candidate at
+ * -inf can still be taken when nothing better is left, so picks stay distinct */
+static int argmax_lowest(const double* a, const char* inS, int n) {
+    int best = -1;
+    for (int i = 0; i < n; ++i) {
+        if (inS[i]) continue;
+        if (best < 0 || a[i] > a[best]) best = i;
+    }
     return best;
 }
 
@@ -137,7 +141,7 @@ int orc_select(const double* s_in, const double* sig, int n, int d, int k, doubl
             double pen = (t == 0 || topk_branch) ? 0.0 : lam * m[i];
             a[i] = inS[i] ? -INFINITY : s[i] - pen;
         }
-        int i = argmax_lowest(a, n);
+        int i = argmax_lowest(a, inS, n);
         double sec = second_best(a, n, i);
         order[t] = i;
         gain[t] = a[i];

@@ -120,9 +120,14 @@ def signatures_flat(V_all, eps: float = 1e-8) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- selection
-def _argmax_lowest(a: np.ndarray) -> int:
-    """argmax with ties to the lowest index (np.argmax returns the first maximum)."""
-    return int(np.argmax(a))
+def _argmax_lowest(a: np.ndarray, excluded: Optional[np.ndarray] = None) -> int:
+    """argmax over the candidates not in ``excluded``, ties to the lowest index.
+    (A candidate whose value is -inf can still be taken when nothing better is
+    left, so the result is always a new index.)"""
+    if excluded is None:
+        return int(np.argmax(a))                      # np.argmax returns the first maximum
+    cand = np.nonzero(~excluded)[0]
+    return int(cand[np.argmax(a[cand])])
 
 
 def sanitize_scores(s: np.ndarray):
@@ -178,7 +183,7 @@ def alpha_select(s, sig, k: int, lam: float, force_greedy: bool = False) -> Sele
     order, gains, margins = [], [], []
 
     def pick(a):
-        i = _argmax_lowest(a)
+        i = _argmax_lowest(a, in_S)
         rest = np.delete(a, i)
         second = rest.max() if len(rest) else NEG_INF
         margins.append(a[i] - second if np.isfinite(a[i]) and np.isfinite(second) else
@@ -219,7 +224,9 @@ def alpha_select_gram(s, sig, k: int, lam: float) -> np.ndarray:
     for _t in range(1, k):
         a = s - lam * m
         a[S] = NEG_INF
-        i = _argmax_lowest(a)
+        taken = np.zeros(n, dtype=bool)
+        taken[S] = True
+        i = _argmax_lowest(a, taken)
         S.append(i)
         m = np.maximum(m, Sims[i, :])
     return np.sort(np.array(S, dtype=np.int64))
@@ -296,7 +303,7 @@ def replay_pick_order(s, sig, lam: float, picks: Sequence[int], tol: float = 1e-
             return Replay(False, len(log) + 1, np.inf, log + [(t, i, -1, np.inf)])
         a = s - lam * m if t > 0 else s.copy()
         a[in_S] = NEG_INF
-        best = _argmax_lowest(a)
+        best = _argmax_lowest(a, in_S)
         if best != i:
             deficit = a[best] - a[i] if np.isfinite(a[i]) else (0.0 if not np.isfinite(a[best]) else np.inf)
             log.append((t, i, best, float(deficit)))

@@ -1,0 +1,433 @@
+// Kernels: fused resident event, stand-alone score / select / compact, flat signature (Eq. 1).
+#pragma once
+#include "akv_steps.cuh"
+
+namespace akv {
+
+struct EventArgs {
+    DevLayout lay;
+    void* K;
+    void* V;
+    PosDesc pos;
+    const int* n_cand;      // [B] or null
+    const float* qstat;     // [L,H,d]
+    const int* p_ref;       // [B] or null
+    const float* flat_sig;  // [B,N,d] or null (flat signature mode)
+    int budget;
+    float lam, eps;
+    int greedy;             // 1: run the loop with similarity updates; 0: top-k
+    int* idx_sorted;
+    int* pick_order;
+    float* pick_gain;
+    float* scores;          // in (select) / out (score, fused)
+    int* n_kept;
+    int* status;
+};
+
+__device__ __forceinline__ int event_n(const EventArgs& a, int b) {
+    int n = a.n_cand ? a.n_cand[b] : a.lay.N;
+    return n < 0 ? 0 : (n > a.lay.N ? a.lay.N : n);
+}
+
+__device__ __forceinline__ const int* event_pos(const PosDesc& p, const EventId& id) {
+    return p.p ? p.p + id.b * p.sb + id.l * p.sl + id.h * p.sh : nullptr;
+}
+
+// block-wide max of int values (all threads call); scratch: kWarps ints
+__device__ __forceinline__ int block_max_int(int v, int* scratch) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) r = max(r, scratch[w]);
+    return r;
+}
+
+// Shared-memory carve-up used by the per-event kernels. Offsets in bytes, 16-byte aligned blocks.
+struct SmemPlan {
+    unsigned tileK, tileV, phi, g, pos, s, r, m, order, gain, idx, taken, red, total;
+};
+__host__ __device__ inline unsigned align16(unsigned x) { return (x + 15u) & ~15u; }
+__host__ __device__ inline SmemPlan plan_smem(int N, int d, int esize, int budget, bool withK, bool withV) {
+    SmemPlan p;
+    unsigned o = 0;
+    p.tileK = o; o += withK ? align16((unsigned)N * d * esize) : 0;
+    p.tileV = o; o += withV ? align16((unsigned)N * d * esize) : 0;
+    p.phi = o;   o += align16((unsigned)(d / 2) * 8);
+    p.g = o;     o += align16((unsigned)(d / 2) * 8);
+    p.pos = o;   o += align16((unsigned)N * 4);
+    p.s = o;     o += align16((unsigned)N * 4);
+    p.r = o;     o += align16((unsigned)N * 4);
+    p.m = o;     o += align16((unsigned)N * 4);
+    p.order = o; o += align16((unsigned)budget * 4);
+    p.gain = o;  o += align16((unsigned)budget * 4);
+    p.idx = o;   o += align16((unsigned)budget * 4);
+    p.taken = o; o += align16((unsigned)N);
+    p.red = o;   o += align16(2u * kWarps * 8u + kWarps * 4u);
+    p.total = o;
+    return p;
+}
+
+// copy n rows of one event between global memory and a dense shared tile, 16 bytes per thread and step
+template <typename T>
+__device__ __forceinline__ void load_tile(T* tile, const T* base, const DevLayout& lay, const EventId& id, int n) {
+    const int cpr = lay.d * (int)sizeof(T) / 16;  // 16-byte chunks per row
+    for (int x = threadIdx.x; x < n * cpr; x += kThreads) {
+        const int row = x / cpr, c = x - row * cpr;
+        const char* src = reinterpret_cast<const char*>(base + row_offset(lay, id.b, id.l, id.h, row)) + c * 16;
+        copy16(reinterpret_cast<char*>(tile) + (size_t)x * 16, src);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fused event, tiles resident in shared memory: K and V are read from HBM once and the kept rows
+// are written once. One CTA per (sequence, layer, KV head).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int n = event_n(a, id.b);
+    const int d = lay.d, N = lay.N;
+    const SmemPlan sp = plan_smem(N, d, sizeof(T), a.budget, true, true);
+    T* Kt = reinterpret_cast<T*>(smem + sp.tileK);
+    T* Vt = reinterpret_cast<T*>(smem + sp.tileV);
+    unsigned long long* phi = reinterpret_cast<unsigned long long*>(smem + sp.phi);
+    float2* g = reinterpret_cast<float2*>(smem + sp.g);
+    int* spos = reinterpret_cast<int*>(smem + sp.pos);
+    float* s = reinterpret_cast<float*>(smem + sp.s);
+    float* r = reinterpret_cast<float*>(smem + sp.r);
+    float* m = reinterpret_cast<float*>(smem + sp.m);
+    int* order = reinterpret_cast<int*>(smem + sp.order);
+    float* gain = reinterpret_cast<float*>(smem + sp.gain);
+    int* idx = reinterpret_cast<int*>(smem + sp.idx);
+    unsigned char* taken = smem + sp.taken;
+    unsigned long long* red = reinterpret_cast<unsigned long long*>(smem + sp.red);
+    int* redi = reinterpret_cast<int*>(smem + sp.red + 2 * kWarps * 8);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int* gpos = event_pos(a.pos, id);
+    T* Kg = reinterpret_cast<T*>(a.K);
+    T* Vg = reinterpret_cast<T*>(a.V);
+
+    // stage the event on chip
+    load_tile(Kt, Kg, lay, id, n);
+    load_tile(Vt, Vg, lay, id, n);
+    int pmax = INT_MIN;
+    for (int j = tid; j < n; j += kThreads) {
+        const int p = gpos ? gpos[j] : 0;
+        spos[j] = p;
+        pmax = max(pmax, p);
+        taken[j] = 0;
+        m[j] = 0.f;
+    }
+    for (int f = tid; f < d / 2; f += kThreads) phi[f] = tab.phi[f];
+    fold_query(a.qstat + ((long long)id.l * lay.H + id.h) * d, tab, d, g);
+    long long pref = 0;
+    if (gpos) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)block_max_int(pmax, redi) + 1;
+    __syncthreads();
+
+    // scores and reciprocal norms
+    const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
+    const int RPW = 32 / G, grp = lane / G, lig = lane % G;
+    int bad = 0;
+    for (int j0 = warp * RPW; j0 < n; j0 += kWarps * RPW) {
+        const int j = j0 + grp;
+        const bool valid = j < n;
+        const long long dist = valid ? pref - (long long)spos[j] : 0;
+        const float sc = score_row(Kt + (size_t)j * d, valid, dist, gpos != nullptr, d, phi, g, lig, G);
+        const float ss = a.flat_sig ? 1.f : sumsq_row(Vt + (size_t)j * d, valid, d, lig, G);
+        if (valid && lig == 0) {
+            if (a.scores) a.scores[(long long)id.e * N + j] = sc;
+            const bool fin = isfinite(sc);
+            bad |= !fin;
+            s[j] = fin ? sc : -INFINITY;
+            r[j] = 1.f / (sqrtf(ss) + a.eps);
+        }
+    }
+    bad = __syncthreads_or(bad);
+
+    // selection
+    const int picks = min(a.budget, n);
+    if (a.flat_sig) {
+        StridedRows<float> rows{a.flat_sig + (long long)id.b * N * d, d};
+        greedy_cta<float>(n, picks, a.lam, a.greedy != 0, d, s, nullptr, m, taken, order, gain, rows, red);
+    } else {
+        StridedRows<T> rows{Vt, d};
+        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, rows, red);
+    }
+    ordered_indices(n, a.budget, taken, idx);
+    __syncthreads();
+
+    // outputs
+    const long long ob = (long long)id.e * a.budget;
+    for (int t = tid; t < a.budget; t += kThreads) {
+        a.idx_sorted[ob + t] = idx[t];
+        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
+        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
+    }
+    if (tid == 0) {
+        if (a.n_kept) a.n_kept[id.e] = picks;
+        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+    }
+    // compaction: kept rows go to slots 0..picks-1 of the same buffer (all sources are on chip)
+    const int cpr = d * (int)sizeof(T) / 16;
+    for (int x = tid; x < picks * cpr; x += kThreads) {
+        const int rr = x / cpr, c = x - rr * cpr;
+        const int src = idx[rr];
+        const long long off = row_offset(lay, id.b, id.l, id.h, rr);
+        copy16(reinterpret_cast<char*>(Kg + off) + c * 16, reinterpret_cast<const char*>(Kt + (size_t)src * d) + c * 16);
+        copy16(reinterpret_cast<char*>(Vg + off) + c * 16, reinterpret_cast<const char*>(Vt + (size_t)src * d) + c * 16);
+    }
+    if (gpos) {
+        int* wpos = a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh;
+        for (int t = tid; t < picks; t += kThreads) wpos[t] = spos[idx[t]];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stand-alone score: grid (row blocks, events); K streamed from global memory once.
+// ---------------------------------------------------------------------------------------------
+constexpr int kScoreRows = 64;  // rows per CTA
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+    __shared__ unsigned long long phi[kMaxHalf];
+    __shared__ float2 g[kMaxHalf];
+    __shared__ int redi[kWarps];
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.y);
+    const int n = event_n(a, id.b);
+    const int d = lay.d;
+    const int row0 = blockIdx.x * kScoreRows;
+    if (row0 >= n) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int* gpos = event_pos(a.pos, id);
+    for (int f = tid; f < d / 2; f += kThreads) phi[f] = tab.phi[f];
+    fold_query(a.qstat + ((long long)id.l * lay.H + id.h) * d, tab, d, g);
+    long long pref = 0;
+    if (gpos) {
+        if (a.p_ref) pref = a.p_ref[id.b];
+        else {
+            int pmax = INT_MIN;
+            for (int j = tid; j < n; j += kThreads) pmax = max(pmax, gpos[j]);
+            pref = (long long)block_max_int(pmax, redi) + 1;
+        }
+    }
+    __syncthreads();
+    const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
+    const int RPW = 32 / G, grp = lane / G, lig = lane % G;
+    const T* Kg = reinterpret_cast<const T*>(a.K);
+    int bad = 0;
+    const int rend = min(n, row0 + kScoreRows);
+    for (int j0 = row0 + warp * RPW; j0 < rend; j0 += kWarps * RPW) {
+        const int j = j0 + grp;
+        const bool valid = j < rend;
+        const long long dist = (valid && gpos) ? pref - (long long)gpos[j] : 0;
+        const T* krow = Kg + (valid ? row_offset(lay, id.b, id.l, id.h, j) : 0);
+        const float sc = score_row(krow, valid, dist, gpos != nullptr, d, phi, g, lig, G);
+        if (valid && lig == 0) {
+            a.scores[(long long)id.e * lay.N + j] = sc;
+            bad |= !isfinite(sc);
+        }
+    }
+    if (a.status) {
+        bad = __syncthreads_or(bad);
+        if (tid == 0 && bad) atomicMax(a.status + id.e, 1);
+    }
+}
+
+// zero a status array before the score kernel's atomicMax
+__global__ void fill_int_kernel(int* p, long long n, int v) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stand-alone selection: scores in, indices out. One CTA per event. RESIDENT: the V tile is staged
+// in shared memory; otherwise similarity rows are read from global memory at every step.
+// ---------------------------------------------------------------------------------------------
+template <typename T, bool RESIDENT>
+__global__ void __launch_bounds__(kThreads) select_kernel(const EventArgs a) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int n = event_n(a, id.b);
+    const int d = lay.d, N = lay.N;
+    const SmemPlan sp = plan_smem(N, d, sizeof(T), a.budget, false, RESIDENT);
+    T* Vt = reinterpret_cast<T*>(smem + sp.tileV);
+    float* s = reinterpret_cast<float*>(smem + sp.s);
+    float* r = reinterpret_cast<float*>(smem + sp.r);
+    float* m = reinterpret_cast<float*>(smem + sp.m);
+    int* order = reinterpret_cast<int*>(smem + sp.order);
+    float* gain = reinterpret_cast<float*>(smem + sp.gain);
+    int* idx = reinterpret_cast<int*>(smem + sp.idx);
+    unsigned char* taken = smem + sp.taken;
+    unsigned long long* red = reinterpret_cast<unsigned long long*>(smem + sp.red);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T* Vg = reinterpret_cast<const T*>(a.V);
+    const bool flat = a.flat_sig != nullptr;
+    const bool needV = a.greedy && !flat;
+
+    if (RESIDENT && needV) load_tile(Vt, Vg, lay, id, n);
+    int bad = 0;
+    for (int j = tid; j < n; j += kThreads) {
+        const float sc = a.scores[(long long)id.e * N + j];
+        const bool fin = isfinite(sc);
+        bad |= !fin;
+        s[j] = fin ? sc : -INFINITY;
+        taken[j] = 0;
+        m[j] = 0.f;
+    }
+    bad = __syncthreads_or(bad);
+    LayoutRows<T> grows{Vg, &lay, id.b, id.l, id.h};
+    StridedRows<T> srows{Vt, d};
+    if (needV) {
+        const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
+        const int RPW = 32 / G, grp = lane / G, lig = lane % G;
+        for (int j0 = warp * RPW; j0 < n; j0 += kWarps * RPW) {
+            const int j = j0 + grp;
+            const bool valid = j < n;
+            const T* row = RESIDENT ? srows(valid ? j : 0) : grows(valid ? j : 0);
+            const float ss = sumsq_row(row, valid, d, lig, G);
+            if (valid && lig == 0) r[j] = 1.f / (sqrtf(ss) + a.eps);
+        }
+        __syncthreads();
+    }
+    const int picks = min(a.budget, n);
+    if (flat) {
+        StridedRows<float> rows{a.flat_sig + (long long)id.b * N * d, d};
+        greedy_cta<float>(n, picks, a.lam, a.greedy != 0, d, s, nullptr, m, taken, order, gain, rows, red);
+    } else if (RESIDENT) {
+        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, srows, red);
+    } else {
+        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, grows, red);
+    }
+    ordered_indices(n, a.budget, taken, idx);
+    __syncthreads();
+    const long long ob = (long long)id.e * a.budget;
+    for (int t = tid; t < a.budget; t += kThreads) {
+        a.idx_sorted[ob + t] = idx[t];
+        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
+        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
+    }
+    if (tid == 0) {
+        if (a.n_kept) a.n_kept[id.e] = picks;
+        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stand-alone compaction, in place. Rows move in ascending chunks staged through shared memory:
+// a chunk's destinations [c0, c1) can only overlap sources of the same chunk (idx[r] >= r and idx
+// ascending), which are on chip before the first store.
+// ---------------------------------------------------------------------------------------------
+struct CompactArgs {
+    DevLayout lay;
+    void* K;
+    void* V;
+    PosDesc pos;
+    const int* idx_sorted;
+    int budget;
+    int chunk_rows;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) compact_kernel(const CompactArgs a) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int d = lay.d;
+    const int tid = threadIdx.x;
+    const int rowB = d * (int)sizeof(T);
+    const int cpr = rowB / 16;
+    unsigned char* stK = smem;
+    unsigned char* stV = smem + (size_t)a.chunk_rows * rowB;
+    int* sidx = reinterpret_cast<int*>(smem + 2 * (size_t)a.chunk_rows * rowB);
+    int* spos = sidx + a.chunk_rows;
+    const int* gidx = a.idx_sorted + (long long)id.e * a.budget;
+    T* Kg = reinterpret_cast<T*>(a.K);
+    T* Vg = reinterpret_cast<T*>(a.V);
+    int* gpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
+    for (int c0 = 0; c0 < a.budget; c0 += a.chunk_rows) {
+        const int cn = min(a.chunk_rows, a.budget - c0);
+        __syncthreads();
+        for (int t = tid; t < cn; t += kThreads) {
+            const int src = gidx[c0 + t];
+            sidx[t] = (src >= 0 && src < lay.N) ? src : -1;
+            if (gpos && sidx[t] >= 0) spos[t] = gpos[src];
+        }
+        __syncthreads();
+        for (int x = tid; x < cn * cpr; x += kThreads) {
+            const int rr = x / cpr, c = x - rr * cpr;
+            const int src = sidx[rr];
+            if (src < 0) continue;
+            const long long off = row_offset(lay, id.b, id.l, id.h, src);
+            if (Kg) copy16(stK + (size_t)x * 16, reinterpret_cast<const char*>(Kg + off) + c * 16);
+            if (Vg) copy16(stV + (size_t)x * 16, reinterpret_cast<const char*>(Vg + off) + c * 16);
+        }
+        __syncthreads();
+        for (int x = tid; x < cn * cpr; x += kThreads) {
+            const int rr = x / cpr, c = x - rr * cpr;
+            if (sidx[rr] < 0) continue;
+            const long long off = row_offset(lay, id.b, id.l, id.h, c0 + rr);
+            if (Kg) copy16(reinterpret_cast<char*>(Kg + off) + c * 16, stK + (size_t)x * 16);
+            if (Vg) copy16(reinterpret_cast<char*>(Vg + off) + c * 16, stV + (size_t)x * 16);
+        }
+        if (gpos)
+            for (int t = tid; t < cn; t += kThreads)
+                if (sidx[t] >= 0) gpos[c0 + t] = spos[t];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 1: flat signature. One warp group per (sequence, slot): u = mean over (l, h) of V rows,
+// v = u / (||u|| + eps), written as fp32 [B, N, d].
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) flat_signature_kernel(const DevLayout lay, const void* V, const int* n_cand,
+                                                                 float eps, float* out) {
+    const int d = lay.d;
+    const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
+    const int RPW = 32 / G;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int grp = lane / G, lig = lane % G;
+    const long long slot = ((long long)blockIdx.x * kWarps + warp) * RPW + grp;  // over B*N
+    const bool inrange = slot < (long long)lay.B * lay.N;
+    const int b = inrange ? (int)(slot / lay.N) : 0;
+    const int j = inrange ? (int)(slot % lay.N) : 0;
+    int n = n_cand ? n_cand[b] : lay.N;
+    n = n < 0 ? 0 : (n > lay.N ? lay.N : n);
+    const bool valid = inrange && j < n;
+    const bool act = valid && lig * 8 < d;
+    const T* Vg = reinterpret_cast<const T*>(V);
+    float u[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (act) {
+        for (int l = 0; l < lay.L; ++l)
+            for (int h = 0; h < lay.H; ++h) {
+                float x[8];
+                load8(Vg + row_offset(lay, b, l, h, j) + lig * 8, x);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) u[q] += x[q];
+            }
+        const float inv = 1.f / (float)(lay.L * lay.H);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) u[q] *= inv;
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) ss = fmaf(u[q], u[q], ss);
+    ss = group_sum(ss, G);
+    if (act) {
+        const float r = 1.f / (sqrtf(ss) + eps);
+        float* o = out + slot * d + lig * 8;
+        *reinterpret_cast<float4*>(o) = make_float4(u[0] * r, u[1] * r, u[2] * r, u[3] * r);
+        *reinterpret_cast<float4*>(o + 4) = make_float4(u[4] * r, u[5] * r, u[6] * r, u[7] * r);
+    }
+}
+
+}  // namespace akv

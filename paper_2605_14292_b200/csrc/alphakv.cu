@@ -1,0 +1,460 @@
+// C ABI of the alphakv library: argument validation, table set-up and kernel launches.
+#include "../../include/alphakv.h"
+
+#include <atomic>
+#include <climits>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "akv_kernels.cuh"
+
+using namespace akv;
+
+struct akv_handle {
+    int device;
+    int smem_optin;    // largest dynamic shared memory per CTA
+    int sm_count;
+    void* ws;          // grow-only scratch
+    size_t ws_bytes;
+    // cached score tables
+    ScoreTab tab;
+    float tab_base;
+    int tab_d, tab_W;
+};
+
+static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+static akv_status_t fail(akv_status_t s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+#define CUDA_TRY(expr)                                                                             \
+    do {                                                                                           \
+        cudaError_t e_ = (expr);                                                                   \
+        if (e_ != cudaSuccess) return fail(AKV_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+extern "C" const char* akv_last_error(void) { return g_err; }
+extern "C" uint64_t akv_launch_count(void) { return g_launches.load(); }
+extern "C" const char* akv_status_string(akv_status_t s) {
+    switch (s) {
+        case AKV_OK: return "ok";
+        case AKV_ERR_INVALID_ARG: return "invalid argument";
+        case AKV_ERR_UNSUPPORTED: return "unsupported";
+        case AKV_ERR_BUDGET: return "budget out of range";
+        case AKV_ERR_ALIGNMENT: return "alignment";
+        case AKV_ERR_WORKSPACE: return "workspace";
+        case AKV_ERR_CUDA: return "cuda error";
+    }
+    return "unknown";
+}
+
+extern "C" void akv_default_options(akv_options_t* o) {
+    if (!o) return;
+    o->lambda = 0.5f;
+    o->eps = 1e-8f;
+    o->rope_base = 10000.f;
+    o->future_window = 1;
+    o->sig_mode = AKV_SIG_PER_HEAD;
+    o->flags = 0;
+}
+
+extern "C" akv_status_t akv_create(akv_handle_t** out, int device) {
+    if (!out) return fail(AKV_ERR_INVALID_ARG, "akv_create: out is NULL");
+    *out = nullptr;
+    int count = 0;
+    CUDA_TRY(cudaGetDeviceCount(&count));
+    if (device < 0 || device >= count) return fail(AKV_ERR_INVALID_ARG, "akv_create: device %d of %d", device, count);
+    akv_handle* h = new akv_handle();
+    memset(h, 0, sizeof(*h));
+    h->device = device;
+    cudaError_t e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) {
+        delete h;
+        return fail(AKV_ERR_CUDA, "akv_create: %s", cudaGetErrorString(e));
+    }
+    h->tab_d = -1;
+    *out = h;
+    return AKV_OK;
+}
+
+extern "C" akv_status_t akv_destroy(akv_handle_t* h) {
+    if (!h) return AKV_OK;
+    if (h->ws) {
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(h->device);
+        cudaFree(h->ws);
+        cudaSetDevice(prev);
+    }
+    delete h;
+    return AKV_OK;
+}
+
+static akv_status_t workspace(akv_handle* h, size_t bytes, void** out) {
+    if (bytes > h->ws_bytes) {
+        if (h->ws) {
+            CUDA_TRY(cudaDeviceSynchronize());  // earlier launches may still use the old buffer
+            CUDA_TRY(cudaFree(h->ws));
+            h->ws = nullptr;
+            h->ws_bytes = 0;
+        }
+        size_t want = (bytes + (size_t(1) << 20) - 1) & ~((size_t(1) << 20) - 1);
+        if (cudaMalloc(&h->ws, want) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(AKV_ERR_WORKSPACE, "cannot allocate %zu bytes of scratch", want);
+        }
+        h->ws_bytes = want;
+    }
+    *out = h->ws;
+    return AKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// validation
+// ------------------------------------------------------------------------------------------------
+static bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static akv_status_t check_layout(const akv_layout_t* y, DevLayout* out) {
+    if (!y) return fail(AKV_ERR_INVALID_ARG, "layout is NULL");
+    if (y->B < 1 || y->L < 1 || y->H < 1 || y->N < 1 || y->d < 1)
+        return fail(AKV_ERR_INVALID_ARG, "layout: B, L, H, N, d must be positive (got %d %d %d %d %d)", y->B, y->L, y->H,
+                    y->N, y->d);
+    if (y->dtype != AKV_F32 && y->dtype != AKV_BF16) return fail(AKV_ERR_UNSUPPORTED, "layout: dtype %d", (int)y->dtype);
+    if (y->d % 8 != 0 || y->d > kMaxD) return fail(AKV_ERR_UNSUPPORTED, "layout: d = %d must be a multiple of 8, <= %d", y->d, kMaxD);
+    if ((long long)y->B * y->L * y->H > INT_MAX) return fail(AKV_ERR_UNSUPPORTED, "layout: too many events");
+    const long long es = y->dtype == AKV_BF16 ? 2 : 4;
+    DevLayout o;
+    memset(&o, 0, sizeof(o));
+    o.B = y->B; o.L = y->L; o.H = y->H; o.N = y->N; o.d = y->d;
+    o.dtype = (int)y->dtype;
+    o.sl = y->stride_l;
+    if (y->page_size == 0) {
+        o.sb = y->stride_b; o.sh = y->stride_h; o.sn = y->stride_n;
+        if (o.sn < y->d) return fail(AKV_ERR_INVALID_ARG, "layout: stride_n %lld < d", o.sn);
+        const long long st[4] = {o.sb, o.sl, o.sh, o.sn};
+        for (long long s : st)
+            if (s < 0 || (s * es) % 16 != 0) return fail(AKV_ERR_ALIGNMENT, "layout: stride %lld elements is not a multiple of 16 bytes", s);
+    } else {
+        if (!is_pow2(y->page_size)) return fail(AKV_ERR_INVALID_ARG, "layout: page_size %d is not a power of two", y->page_size);
+        if (!y->block_table) return fail(AKV_ERR_INVALID_ARG, "layout: paged but block_table is NULL");
+        if (y->pages_per_seq < 1 || (long long)y->pages_per_seq * y->page_size < y->N)
+            return fail(AKV_ERR_INVALID_ARG, "layout: N = %d exceeds pages_per_seq * page_size", y->N);
+        o.page_size = y->page_size;
+        o.page_shift = 0;
+        while ((1 << o.page_shift) < y->page_size) ++o.page_shift;
+        o.table = y->block_table;
+        o.pps = y->pages_per_seq;
+        o.s_page = y->stride_page; o.s_page_h = y->stride_page_h; o.s_page_n = y->stride_page_n;
+        if (o.s_page_n < y->d) return fail(AKV_ERR_INVALID_ARG, "layout: stride_page_n %lld < d", o.s_page_n);
+        const long long st[4] = {o.sl, o.s_page, o.s_page_h, o.s_page_n};
+        for (long long s : st)
+            if (s < 0 || (s * es) % 16 != 0) return fail(AKV_ERR_ALIGNMENT, "layout: stride %lld elements is not a multiple of 16 bytes", s);
+    }
+    *out = o;
+    return AKV_OK;
+}
+
+static akv_status_t check_options(const akv_options_t* o) {
+    if (!o) return fail(AKV_ERR_INVALID_ARG, "options is NULL");
+    if (!(o->lambda >= 0.f) || !std::isfinite(o->lambda)) return fail(AKV_ERR_INVALID_ARG, "lambda must be finite and >= 0");
+    if (!(o->eps >= 0.f) || !std::isfinite(o->eps)) return fail(AKV_ERR_INVALID_ARG, "eps must be finite and >= 0");
+    if (!(o->rope_base > 0.f) || !std::isfinite(o->rope_base)) return fail(AKV_ERR_INVALID_ARG, "rope_base must be positive");
+    if (o->future_window < 1 || o->future_window > 65536) return fail(AKV_ERR_INVALID_ARG, "future_window must be in 1..65536");
+    if (o->sig_mode != AKV_SIG_PER_HEAD && o->sig_mode != AKV_SIG_FLAT) return fail(AKV_ERR_UNSUPPORTED, "sig_mode %d", (int)o->sig_mode);
+    return AKV_OK;
+}
+
+static akv_status_t check_budget(int budget, int N) {
+    if (budget < 1 || budget > N) return fail(AKV_ERR_BUDGET, "budget %d outside 1..N (N = %d)", budget, N);
+    return AKV_OK;
+}
+
+static akv_status_t check_pos_written(const DevLayout& y, const int32_t* pos, int64_t sb, int64_t sl, int64_t sh) {
+    if (!pos) return AKV_OK;
+    if ((y.B > 1 && sb == 0) || (y.L > 1 && sl == 0) || (y.H > 1 && sh == 0))
+        return fail(AKV_ERR_INVALID_ARG, "pos is rewritten per event: its (b, l, h) strides must not broadcast");
+    return AKV_OK;
+}
+
+// phi[f] = frac(theta_f / 2 pi) in 0.64 fixed point; cw[f] = mean_w exp(i w theta_f)
+static void build_tables(akv_handle* h, int d, float base, int W) {
+    if (h->tab_d == d && h->tab_base == base && h->tab_W == W) return;
+    const long double two_pi = 6.283185307179586476925286766559L;
+    for (int f = 0; f < d / 2; ++f) {
+        const long double theta = powl((long double)base, -2.0L * f / d);
+        long double turns = theta / two_pi;
+        turns -= floorl(turns);
+        h->tab.phi[f] = (unsigned long long)ldexpl(turns, 64);
+        double cr = 0.0, ci = 0.0;
+        for (int w = 0; w < W; ++w) {
+            cr += cos((double)(w * theta));
+            ci += sin((double)(w * theta));
+        }
+        h->tab.cw[f] = make_float2((float)(cr / W), (float)(ci / W));
+    }
+    for (int f = d / 2; f < kMaxHalf; ++f) {
+        h->tab.phi[f] = 0;
+        h->tab.cw[f] = make_float2(0.f, 0.f);
+    }
+    h->tab_d = d; h->tab_base = base; h->tab_W = W;
+}
+
+template <typename K>
+static akv_status_t set_smem(K kernel, unsigned bytes) {
+    if (bytes > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return AKV_OK;
+}
+
+static akv_status_t launched(const char* what) {
+    g_launches.fetch_add(1);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(AKV_ERR_CUDA, "%s launch: %s", what, cudaGetErrorString(e));
+    return AKV_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// ------------------------------------------------------------------------------------------------
+// launch helpers
+// ------------------------------------------------------------------------------------------------
+static akv_status_t launch_score(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    if (a.status) {
+        fill_int_kernel<<<(E + 255) / 256, 256, 0, st>>>(a.status, E, 0);
+        akv_status_t s = launched("fill");
+        if (s != AKV_OK) return s;
+    }
+    dim3 grid((a.lay.N + kScoreRows - 1) / kScoreRows, E);
+    if (a.lay.dtype == AKV_BF16) score_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(a, h->tab);
+    else score_kernel<float><<<grid, kThreads, 0, st>>>(a, h->tab);
+    return launched("score");
+}
+
+template <typename T>
+static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    const bool needV = a.greedy && !a.flat_sig;
+    const SmemPlan res = plan_smem(a.lay.N, a.lay.d, sizeof(T), a.budget, false, true);
+    const SmemPlan non = plan_smem(a.lay.N, a.lay.d, sizeof(T), a.budget, false, false);
+    if (needV && (int)res.total <= h->smem_optin) {
+        akv_status_t s = set_smem(select_kernel<T, true>, res.total);
+        if (s != AKV_OK) return s;
+        select_kernel<T, true><<<E, kThreads, res.total, st>>>(a);
+    } else {
+        if ((int)non.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "N = %d is too large for the selection kernel", a.lay.N);
+        akv_status_t s = set_smem(select_kernel<T, false>, non.total);
+        if (s != AKV_OK) return s;
+        select_kernel<T, false><<<E, kThreads, non.total, st>>>(a);
+    }
+    return launched("select");
+}
+static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st) : launch_select_t<float>(h, a, st);
+}
+
+static akv_status_t launch_compact(akv_handle* h, const CompactArgs& a0, cudaStream_t st) {
+    CompactArgs a = a0;
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    const int rowB = a.lay.d * (a.lay.dtype == AKV_BF16 ? 2 : 4);
+    int rows = (64 * 1024) / (2 * rowB + 8);
+    if (rows > a.budget) rows = a.budget;
+    if (rows < 1) rows = 1;
+    a.chunk_rows = rows;
+    const unsigned bytes = (unsigned)rows * (2 * rowB + 8);
+    if (a.lay.dtype == AKV_BF16) {
+        akv_status_t s = set_smem(compact_kernel<__nv_bfloat16>, bytes);
+        if (s != AKV_OK) return s;
+        compact_kernel<__nv_bfloat16><<<E, kThreads, bytes, st>>>(a);
+    } else {
+        akv_status_t s = set_smem(compact_kernel<float>, bytes);
+        if (s != AKV_OK) return s;
+        compact_kernel<float><<<E, kThreads, bytes, st>>>(a);
+    }
+    (void)h;
+    return launched("compact");
+}
+
+// ------------------------------------------------------------------------------------------------
+// entry points
+// ------------------------------------------------------------------------------------------------
+extern "C" akv_status_t alpha_score(akv_handle_t* h, const akv_layout_t* lay, const void* K, const int32_t* pos,
+                                    int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand, const float* qstat,
+                                    const int32_t* p_ref, const akv_options_t* opt, float* scores, int32_t* status,
+                                    void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_score: handle is NULL");
+    EventArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if (!K || !qstat || !scores) return fail(AKV_ERR_INVALID_ARG, "alpha_score: K, qstat and scores must not be NULL");
+    if (!aligned16(K)) return fail(AKV_ERR_ALIGNMENT, "alpha_score: K is not 16-byte aligned");
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    build_tables(h, lay->d, opt->rope_base, opt->future_window);
+    a.K = const_cast<void*>(K);
+    a.pos = PosDesc{const_cast<int*>(pos), psb, psl, psh};
+    a.n_cand = n_cand; a.qstat = qstat; a.p_ref = p_ref;
+    a.scores = scores; a.status = status;
+    return launch_score(h, a, (cudaStream_t)stream);
+}
+
+static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, const void* V, const float* flat_sig) {
+    a.lam = opt->lambda;
+    a.eps = opt->eps;
+    a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
+    if (opt->sig_mode == AKV_SIG_FLAT) {
+        if (!flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat signature mode needs flat_sig");
+        if (!aligned16(flat_sig)) return fail(AKV_ERR_ALIGNMENT, "flat_sig is not 16-byte aligned");
+        a.flat_sig = flat_sig;
+    } else {
+        if (flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat_sig given but sig_mode is per-head");
+        if (a.greedy && !V) return fail(AKV_ERR_INVALID_ARG, "V must not be NULL in per-head signature mode");
+    }
+    return AKV_OK;
+}
+
+extern "C" akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, const float* scores, const void* V,
+                                     const float* flat_sig, const int32_t* n_cand, int32_t budget,
+                                     const akv_options_t* opt, int32_t* idx_sorted, int32_t* pick_order,
+                                     float* pick_gain, int32_t* n_kept, int32_t* status, void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_select: handle is NULL");
+    EventArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if ((s = check_budget(budget, lay->N)) != AKV_OK) return s;
+    if (!scores || !idx_sorted) return fail(AKV_ERR_INVALID_ARG, "alpha_select: scores and idx_sorted must not be NULL");
+    if (V && !aligned16(V)) return fail(AKV_ERR_ALIGNMENT, "alpha_select: V is not 16-byte aligned");
+    if ((s = fill_select_args(a, opt, V, flat_sig)) != AKV_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    a.V = const_cast<void*>(V);
+    a.n_cand = n_cand;
+    a.budget = budget;
+    a.scores = const_cast<float*>(scores);
+    a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
+    a.n_kept = n_kept; a.status = status;
+    return launch_select(h, a, (cudaStream_t)stream);
+}
+
+extern "C" akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+                                             const int32_t* n_cand, const akv_options_t* opt, float* flat_sig,
+                                             void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_signature_flat: handle is NULL");
+    DevLayout y;
+    akv_status_t s = check_layout(lay, &y);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if (!V || !flat_sig) return fail(AKV_ERR_INVALID_ARG, "alpha_signature_flat: V and flat_sig must not be NULL");
+    if (!aligned16(V) || !aligned16(flat_sig)) return fail(AKV_ERR_ALIGNMENT, "alpha_signature_flat: pointers must be 16-byte aligned");
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    const int G = pow2_ceil(y.d >> 3) > 32 ? 32 : pow2_ceil(y.d >> 3);
+    const long long per_cta = (long long)kWarps * (32 / G);
+    const long long slots = (long long)y.B * y.N;
+    const unsigned grid = (unsigned)((slots + per_cta - 1) / per_cta);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (y.dtype == AKV_BF16) flat_signature_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig);
+    else flat_signature_kernel<float><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig);
+    return launched("flat_signature");
+}
+
+extern "C" akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                   int64_t psb, int64_t psl, int64_t psh, const int32_t* idx_sorted, int32_t budget,
+                                   void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "kv_compact: handle is NULL");
+    CompactArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_budget(budget, lay->N)) != AKV_OK) return s;
+    if (!idx_sorted) return fail(AKV_ERR_INVALID_ARG, "kv_compact: idx_sorted is NULL");
+    if ((K && !aligned16(K)) || (V && !aligned16(V))) return fail(AKV_ERR_ALIGNMENT, "kv_compact: K/V must be 16-byte aligned");
+    if ((s = check_pos_written(a.lay, pos, psb, psl, psh)) != AKV_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    a.K = K; a.V = V;
+    a.pos = PosDesc{pos, psb, psl, psh};
+    a.idx_sorted = idx_sorted;
+    a.budget = budget;
+    return launch_compact(h, a, (cudaStream_t)stream);
+}
+
+extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                             int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand,
+                                             const float* qstat, const int32_t* p_ref, const float* flat_sig,
+                                             int32_t budget, const akv_options_t* opt, int32_t* idx_sorted,
+                                             int32_t* pick_order, float* pick_gain, float* scores, int32_t* n_kept,
+                                             int32_t* status, void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_compress_event: handle is NULL");
+    EventArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if ((s = check_budget(budget, lay->N)) != AKV_OK) return s;
+    if (!K || !V || !qstat || !idx_sorted)
+        return fail(AKV_ERR_INVALID_ARG, "alpha_compress_event: K, V, qstat and idx_sorted must not be NULL");
+    if (!aligned16(K) || !aligned16(V)) return fail(AKV_ERR_ALIGNMENT, "alpha_compress_event: K/V must be 16-byte aligned");
+    if ((s = check_pos_written(a.lay, pos, psb, psl, psh)) != AKV_OK) return s;
+    if ((s = fill_select_args(a, opt, V, flat_sig)) != AKV_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    build_tables(h, lay->d, opt->rope_base, opt->future_window);
+    cudaStream_t st = (cudaStream_t)stream;
+    a.K = K; a.V = V;
+    a.pos = PosDesc{pos, psb, psl, psh};
+    a.n_cand = n_cand; a.qstat = qstat; a.p_ref = p_ref;
+    a.budget = budget;
+    a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
+    a.scores = scores; a.n_kept = n_kept; a.status = status;
+
+    const int es = lay->dtype == AKV_BF16 ? 2 : 4;
+    const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
+    if ((int)res.total <= h->smem_optin) {
+        const int E = a.lay.B * a.lay.L * a.lay.H;
+        if (lay->dtype == AKV_BF16) {
+            if ((s = set_smem(event_resident_kernel<__nv_bfloat16>, res.total)) != AKV_OK) return s;
+            event_resident_kernel<__nv_bfloat16><<<E, kThreads, res.total, st>>>(a, h->tab);
+        } else {
+            if ((s = set_smem(event_resident_kernel<float>, res.total)) != AKV_OK) return s;
+            event_resident_kernel<float><<<E, kThreads, res.total, st>>>(a, h->tab);
+        }
+        return launched("event");
+    }
+    // The event does not fit on chip: score -> select -> compact as three launches, scores held in
+    // the caller's buffer or in the handle's scratch.
+    if (!a.scores) {
+        void* ws = nullptr;
+        const size_t bytes = (size_t)a.lay.B * a.lay.L * a.lay.H * a.lay.N * sizeof(float);
+        if ((s = workspace(h, bytes, &ws)) != AKV_OK) return s;
+        a.scores = static_cast<float*>(ws);
+    }
+    EventArgs sa = a;
+    sa.status = nullptr;  // the selection kernel writes the final status word
+    if ((s = launch_score(h, sa, st)) != AKV_OK) return s;
+    if ((s = launch_select(h, a, st)) != AKV_OK) return s;
+    CompactArgs c;
+    memset(&c, 0, sizeof(c));
+    c.lay = a.lay; c.K = K; c.V = V; c.pos = a.pos; c.idx_sorted = idx_sorted; c.budget = budget;
+    return launch_compact(h, c, st);
+}

@@ -1,0 +1,120 @@
+"""The five benchmark configurations against the oracle (full size where the oracle finishes in
+seconds, sampled events otherwise)."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+import paper_2605_14292_b200 as akv
+from oracle import alpha_oracle as O
+from oracle import c_oracle as CO
+from paper_2605_14292_b200 import synth
+
+import akv_check as chk
+from test_gpu_parity import check_all, dev, run_fused
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+@pytest.mark.parametrize("lam", [0.5, 0.0, 1.0])
+def test_c1_single_event_fp32(lam):
+    ev = synth.make_c1()
+    g = run_fused(ev, lam=lam)
+    log = check_all(ev, g, lam)
+    print("C1 lambda", lam, "near-tie divergences:", log)
+
+
+def test_c2_qwen7b_shaped():
+    ev = synth.make_c2()
+    g = run_fused(ev)
+    log = check_all(ev, g, ev.lam)
+    print("C2 near-tie divergences:", log)
+
+
+def test_c3_llama8b_shaped_full_batch():
+    ev = synth.make_c3()
+    g = run_fused(ev)
+    log = check_all(ev, g, ev.lam)
+    print("C3 near-tie divergences (step, gpu pick, oracle pick, deficit):", log)
+    assert len(log) < 200
+
+
+@pytest.mark.parametrize("lam", [0.0, 0.5, 1.0])
+def test_c4_large_pool_sampled_events(lam):
+    ev = synth.make_c4(B=2, lam=lam)
+    g = run_fused(ev, lam=lam)
+    B, L, H, N, d = ev.shape
+    rng = np.random.default_rng(4)
+    sample = sorted(rng.choice(B * L * H, size=12, replace=False).tolist())
+    log = check_all(ev, g, lam, events=sample)
+    print("C4 lambda", lam, "near-tie divergences:", log)
+    if lam == 0.0:
+        for e in sample:
+            b, l, h = e // (L * H), (e // H) % L, e % H
+            s = g["scores"][b, l, h].astype(np.float64)
+            assert g["idx"][b, l, h].tolist() == np.sort(O.topk_indices(s, ev.budget)).tolist()
+
+
+def _c5_round(c5, pool_K, pool_V, pos, table, q, lay, opts, sel):
+    akv.alpha_compress_event(pool_K, pool_V, pos, q, c5.budget, opts, layout=lay, out=sel)
+
+
+@pytest.mark.parametrize("B,rounds,n_sample", [(4, 3, None), (64, 32, 24)])
+def test_c5_decode_cadence_paged(B, rounds, n_sample):
+    c5 = synth.make_c5(B=B, rounds=rounds)
+    L, H, N, d, b = c5.L, c5.H, c5.N, c5.d, c5.budget
+    E = B * L * H
+    rng = np.random.default_rng(5)
+    sample = list(range(E)) if n_sample is None else sorted(rng.choice(E, size=n_sample, replace=False).tolist())
+    pool_K, pool_V = dev(c5.pool_K), dev(c5.pool_V)
+    table, pos, q = dev(c5.block_table), dev(c5.pos), dev(c5.qstat)
+    rK, rV = dev(c5.refill_K), dev(c5.refill_V)
+    lay = akv.Layout.paged(pool_K, table)
+    opts = akv.Options(lam=c5.lam)
+    # host mirror of the sampled heads, advanced by the oracle
+    hostK = synth.paged_gather_dense(c5.pool_K, c5.block_table)
+    hostV = synth.paged_gather_dense(c5.pool_V, c5.block_table)
+    mirror = {}
+    for e in sample:
+        bb, l, h = e // (L * H), (e // H) % L, e % H
+        mirror[e] = [hostK[bb, l, h].copy(), hostV[bb, l, h].copy(), c5.pos[bb, l, h].copy()]
+    del hostK, hostV
+    page_of = table.long()                                           # [B, pps]
+    n_new = N - b
+    slots = torch.arange(b, N, device="cuda")
+    n_logged = 0
+    for r in range(rounds):
+        sel = akv.alpha_compress_event(pool_K, pool_V, pos, q, b, opts, layout=lay, want_scores=True)
+        torch.cuda.synchronize()
+        idx, order, sc = sel.idx_sorted.cpu().numpy(), sel.pick_order.cpu().numpy(), sel.scores.cpu().numpy()
+        # check the sampled heads: gather their post-event rows from the pool
+        posn = pos.cpu().numpy()
+        for e in sample:
+            bb, l, h = e // (L * H), (e // H) % L, e % H
+            pages = c5.block_table[bb]
+            Kn = akv.to_host_bits(pool_K[l, pages.tolist(), h]).reshape(N, d)
+            Vn = akv.to_host_bits(pool_V[l, pages.tolist(), h]).reshape(N, d)
+            mk, mv, mp = mirror[e]
+            log = []
+            chk.check_event(mk, mv, mp, c5.qstat[l, h], None, b, c5.lam, sc[bb, l, h], order[bb, l, h], idx[bb, l, h],
+                            Kn, Vn, posn[bb, l, h], log=log)
+            n_logged += len(log)
+            # advance the mirror with the GPU's (validated) selection, then the refill
+            ii = idx[bb, l, h]
+            blk = r % c5.refill_K.shape[0]
+            mirror[e] = [np.concatenate([mk[ii], c5.refill_K[blk, l, h]]), np.concatenate([mv[ii], c5.refill_V[blk, l, h]]),
+                         np.concatenate([mp[ii], (N + r * n_new + np.arange(n_new)).astype(np.int32)])]
+        # refill slots b..N-1 of every head with the next block (harness work, plain torch indexing)
+        blk = r % rK.shape[0]
+        pg = page_of[:, (slots // c5.page)]                              # [B, n_new]
+        off = (slots % c5.page)[None, :].expand(B, -1)
+        for l in range(L):
+            pool_K[l, pg, :, off] = rK[blk, l].permute(1, 0, 2)[None].expand(B, -1, -1, -1)
+            pool_V[l, pg, :, off] = rV[blk, l].permute(1, 0, 2)[None].expand(B, -1, -1, -1)
+        pos[..., b:] = (N + r * n_new + torch.arange(n_new, device="cuda", dtype=torch.int32))
+    print("C5 near-tie divergences logged:", n_logged)

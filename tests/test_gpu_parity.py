@@ -1,0 +1,261 @@
+"""GPU-vs-oracle parity, through the C ABI (via the thin binding), element by element."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+import paper_2605_14292_b200 as akv
+from oracle import alpha_oracle as O
+from oracle import c_oracle as CO
+from paper_2605_14292_b200 import synth
+
+import akv_check as chk
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+    akv.load_library()
+
+
+def dev(x):
+    return akv.to_device(x, "cuda")
+
+
+def run_fused(ev, lam=None, flags=0, n_cand=None, p_ref=True, W=None):
+    lam = ev.lam if lam is None else lam
+    K, V, pos, q = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat)
+    pref = dev(ev.p_ref) if p_ref else None
+    nc = None if n_cand is None else dev(np.asarray(n_cand, dtype=np.int32))
+    opts = akv.Options(lam=lam, eps=ev.eps, rope_base=ev.rope_base, future_window=W or ev.future_window, flags=flags)
+    sel = akv.alpha_compress_event(K, V, pos, q, ev.budget, opts, p_ref=pref, n_cand=nc, want_scores=True)
+    torch.cuda.synchronize()
+    return dict(K=akv.to_host_bits(K), V=akv.to_host_bits(V), pos=pos.cpu().numpy(), idx=sel.idx_sorted.cpu().numpy(),
+                order=sel.pick_order.cpu().numpy(), gain=sel.pick_gain.cpu().numpy(), scores=sel.scores.cpu().numpy(),
+                n_kept=sel.n_kept.cpu().numpy(), status=sel.status.cpu().numpy())
+
+
+def check_all(ev, g, lam, events=None, n_cand=None, p_ref=True, W=None, threads=8):
+    B, L, H, N, d = ev.shape
+    W = W or ev.future_window
+    E = B * L * H
+    log = []
+    ref = None
+    if n_cand is None and p_ref and events is None:
+        ref = CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lam, W=W, base=ev.rope_base,
+                             eps=ev.eps, threads=threads, want_rows=False)
+    todo = range(E) if events is None else events
+    for e in todo:
+        b, l, h = e // (L * H), (e // H) % L, e % H
+        n = N if n_cand is None else int(n_cand[b])
+        chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h],
+                        int(ev.p_ref[b]) if p_ref else None, ev.budget, lam,
+                        g["scores"][b, l, h], g["order"][b, l, h], g["idx"][b, l, h],
+                        g["K"][b, l, h], g["V"][b, l, h], g["pos"][b, l, h], W=W, base=ev.rope_base, eps=ev.eps,
+                        ref_scores=None if ref is None else ref["scores"][b, l, h],
+                        ref_order=None if ref is None else ref["order"][b, l, h], n=n, log=log)
+        assert g["n_kept"][b, l, h] == min(ev.budget, n)
+        assert g["status"][b, l, h] == (2 if n < ev.budget else 0)
+    return log
+
+
+# ------------------------------------------------------------------ small shapes: several tiles, ragged tails
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
+@pytest.mark.parametrize("N,d,budget", [(100, 128, 37), (77, 64, 77), (192, 128, 64), (33, 16, 5), (130, 256, 40),
+                                        (50, 8, 20), (96, 40, 31)])
+@pytest.mark.parametrize("lam", [0.0, 0.5, 1.5])
+def test_fused_event_small(dtype, N, d, budget, lam):
+    if dtype == synth.F32 and 2 * N * d * 4 > 200_000:
+        pytest.skip("covered by the three-launch path test")
+    ev = synth.make_c3(seed=N + d, B=2, L=2, H=3, N=N, budget=budget) if d == 128 else \
+        synth.make_plain(2, 2, 3, N, d, budget, lam, dtype=dtype, seed=N + d)
+    if d == 128 and dtype == synth.F32:
+        ev = synth.make_plain(2, 2, 3, N, d, budget, lam, dtype=dtype, seed=N + d)
+    g = run_fused(ev, lam=lam)
+    check_all(ev, g, lam)
+
+
+def test_lambda0_greedy_loop_equals_fast_path_equals_topk():
+    ev = synth.make_plain(2, 3, 2, 150, 128, 50, 0.0, dtype=synth.BF16, seed=3)
+    fast = run_fused(ev, lam=0.0)
+    loop = run_fused(ev, lam=0.0, flags=akv.FLAG_FORCE_GREEDY)
+    assert np.array_equal(fast["order"], loop["order"]) and np.array_equal(fast["idx"], loop["idx"])
+    assert np.array_equal(fast["K"][..., :50, :], loop["K"][..., :50, :])
+    # top-k of the GPU's own scores, ties to the lower index
+    for b in range(2):
+        for l in range(3):
+            for h in range(2):
+                s = fast["scores"][b, l, h].astype(np.float64)
+                assert fast["order"][b, l, h].tolist() == O.topk_indices(s, 50).tolist()
+
+
+def test_ragged_candidate_counts_and_short_events():
+    ev = synth.make_plain(4, 2, 2, 120, 128, 40, 0.5, dtype=synth.BF16, seed=9)
+    n_cand = [120, 41, 40, 17]          # last one is below the budget: keep all, status 2
+    g = run_fused(ev, n_cand=n_cand)
+    check_all(ev, g, 0.5, n_cand=n_cand)
+    # rows beyond n_cand were never read as candidates: no index >= n_cand
+    for b, n in enumerate(n_cand):
+        kept = min(40, n)
+        assert g["idx"][b, :, :, :kept].max() < n
+
+
+def test_default_reference_position_and_future_window():
+    ev = synth.make_plain(2, 2, 2, 90, 128, 30, 0.5, dtype=synth.BF16, seed=12)
+    ev.pos[:] = (np.sort(np.random.default_rng(1).choice(5000, size=90, replace=False))).astype(np.int32)
+    g = run_fused(ev, p_ref=False, W=4)
+    check_all(ev, g, 0.5, p_ref=False, W=4)
+
+
+def test_large_positions_keep_score_accuracy():
+    ev = synth.make_plain(1, 2, 2, 64, 128, 16, 0.5, dtype=synth.BF16, seed=13)
+    ev.pos[:] = (1_000_000 + np.arange(64) * 997).astype(np.int32)
+    ev.p_ref[:] = 1_100_000
+    g = run_fused(ev)
+    check_all(ev, g, 0.5)
+
+
+def test_repeat_runs_are_bit_identical():
+    ev = synth.make_c3(seed=4, B=2, L=2, H=2, N=192, budget=64)
+    a, b = run_fused(ev), run_fused(ev)
+    for k in ("K", "V", "pos", "idx", "order", "scores", "gain"):
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_nonfinite_scores_are_flagged_and_never_preferred():
+    ev = synth.make_plain(1, 1, 2, 64, 128, 20, 0.5, dtype=synth.F32, seed=14)
+    ev.K[0, 0, 0, 5, 3] = np.inf
+    ev.K[0, 0, 0, 9, 100] = np.nan
+    g = run_fused(ev)
+    assert g["status"][0, 0, 0] == 1 and g["status"][0, 0, 1] == 0
+    assert not ({5, 9} & set(g["idx"][0, 0, 0].tolist()))
+    assert len(set(g["idx"][0, 0, 0].tolist())) == 20
+
+
+# ------------------------------------------------------------------ stand-alone entry points
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
+def test_score_select_compact_chain_equals_fused(dtype):
+    ev = synth.make_c3(seed=21, B=2, L=2, H=2, N=160, budget=48) if dtype == synth.BF16 else \
+        synth.make_plain(2, 2, 2, 160, 128, 48, 0.5, dtype=dtype, seed=21)
+    fused = run_fused(ev)
+    K, V, pos, q, pref = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    opts = akv.Options(lam=ev.lam)
+    status = torch.full((2, 2, 2), -7, dtype=torch.int32, device="cuda")
+    s = akv.alpha_score(K, q, pos=pos, p_ref=pref, opts=opts, status=status)
+    sel = akv.alpha_select(s, V, ev.budget, opts)
+    akv.kv_compact(K, V, pos, sel.idx_sorted)
+    torch.cuda.synchronize()
+    assert np.array_equal(s.cpu().numpy(), fused["scores"])          # same device code, same bits
+    assert np.array_equal(sel.pick_order.cpu().numpy(), fused["order"])
+    assert np.array_equal(sel.idx_sorted.cpu().numpy(), fused["idx"])
+    assert np.array_equal(sel.pick_gain.cpu().numpy(), fused["gain"])
+    assert np.array_equal(akv.to_host_bits(K)[..., :48, :], fused["K"][..., :48, :])
+    assert np.array_equal(akv.to_host_bits(V)[..., :48, :], fused["V"][..., :48, :])
+    assert np.array_equal(pos.cpu().numpy()[..., :48], fused["pos"][..., :48])
+    assert int(status.abs().max()) == 0
+
+
+def test_score_only_broadcast_positions_and_rotated_cache():
+    ev = synth.make_plain(2, 3, 2, 70, 128, 10, 0.5, dtype=synth.BF16, seed=22)
+    K, q = dev(ev.K), dev(ev.qstat)
+    pos1 = dev(np.arange(70, dtype=np.int32) * 3)
+    s = akv.alpha_score(K, q, pos=pos1, p_ref=dev(np.array([400, 500], dtype=np.int32)),
+                        opts=akv.Options(future_window=3)).cpu().numpy()
+    s0 = akv.alpha_score(K, q, pos=None).cpu().numpy()
+    for b in range(2):
+        for l in range(3):
+            for h in range(2):
+                ref = O.triattention_score(ev.K[b, l, h], np.arange(70) * 3, ev.qstat[l, h], [400, 500][b], 3)
+                chk.check_scores(s[b, l, h], ref, chk.score_scale(ev.K[b, l, h], ev.qstat[l, h], 128))
+                ref0 = O.triattention_score(ev.K[b, l, h], None, ev.qstat[l, h], None)
+                chk.check_scores(s0[b, l, h], ref0, chk.score_scale(ev.K[b, l, h], ev.qstat[l, h], 128))
+
+
+def test_select_given_scores_matches_oracle_and_duplicate_pair_closed_form():
+    P, d = 40, 128
+    s, V, leaders = synth.make_duplicate_pairs(P, d, 0.01, seed=2, dtype=synth.BF16)
+    lam = float(s[0] - 0.01 - s[2 * (P - 1)]) + 0.05
+    sc = torch.tensor(s, dtype=torch.float32, device="cuda").reshape(1, 1, 1, -1).contiguous()
+    Vd = dev(V.reshape(1, 1, 1, 2 * P, d))
+    for b in (1, 7, P):
+        sel = akv.alpha_select(sc, Vd, b, akv.Options(lam=lam))
+        assert sel.idx_sorted.cpu().numpy().ravel().tolist() == leaders[:b].tolist()
+    top = akv.alpha_select(sc, Vd, 6, akv.Options(lam=0.0)).idx_sorted.cpu().numpy().ravel().tolist()
+    assert top == sorted(sorted(range(2 * P), key=lambda i: (-np.float32(s[i]), i))[:6])
+
+
+def test_compact_in_place_aliasing_and_negative_tail():
+    ev = synth.make_plain(2, 2, 2, 64, 128, 20, 0.5, dtype=synth.BF16, seed=23)
+    K, V, pos = dev(ev.K), dev(ev.V), dev(ev.pos)
+    idx = np.zeros((2, 2, 2, 20), dtype=np.int32)
+    idx[...] = np.arange(1, 21)                 # every destination is another row's source
+    idx[1, 1, 1] = np.r_[np.arange(5, 64, 4)[:15], -1, -1, -1, -1, -1]
+    akv.kv_compact(K, V, pos, dev(idx))
+    torch.cuda.synchronize()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    for b in range(2):
+        for l in range(2):
+            for h in range(2):
+                ii = idx[b, l, h]
+                ii = ii[ii >= 0]
+                assert np.array_equal(Kn[b, l, h, :len(ii)], ev.K[b, l, h][ii])
+                assert np.array_equal(Vn[b, l, h, :len(ii)], ev.V[b, l, h][ii])
+                assert np.array_equal(pn[b, l, h, :len(ii)], ev.pos[b, l, h][ii])
+                assert np.array_equal(Kn[b, l, h, 21:], ev.K[b, l, h, 21:])     # untouched beyond the moved range
+
+
+def test_flat_signature_eq1_and_selection_with_it():
+    ev = synth.make_plain(2, 3, 2, 80, 128, 25, 0.7, dtype=synth.BF16, seed=24)
+    V = dev(ev.V)
+    sig = akv.alpha_signature_flat(V).cpu().numpy()
+    for b in range(2):
+        ref = O.signatures_flat(ev.V[b])
+        assert np.max(np.abs(sig[b] - ref)) < 2e-7
+    K, pos, q, pref = dev(ev.K), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    opts = akv.Options(lam=0.7, sig_mode=akv.SIG_FLAT)
+    sel = akv.alpha_compress_event(K, V, pos, q, 25, opts, p_ref=pref, flat_sig=dev(sig), want_scores=True)
+    torch.cuda.synchronize()
+    Kn = akv.to_host_bits(K)
+    for b in range(2):
+        ref_sig = O.signatures_flat(ev.V[b])
+        for l in range(3):
+            for h in range(2):
+                chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]), 25, 0.7,
+                                sel.scores[b, l, h].cpu().numpy(), sel.pick_order[b, l, h].cpu().numpy(),
+                                sel.idx_sorted[b, l, h].cpu().numpy(), Kn[b, l, h], None, None, sig=ref_sig)
+
+
+def test_three_launch_path_for_events_that_do_not_fit_on_chip():
+    """fp32 with N = 600 exceeds shared memory: score -> select -> compact with scratch scores."""
+    ev = synth.make_plain(1, 2, 2, 600, 128, 50, 0.5, dtype=synth.F32, seed=25)
+    K, V, pos, q, pref = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    sel = akv.alpha_compress_event(K, V, pos, q, 50, akv.Options(lam=0.5), p_ref=pref, want_scores=False)
+    torch.cuda.synchronize()
+    g = dict(K=akv.to_host_bits(K), V=akv.to_host_bits(V), pos=pos.cpu().numpy(), idx=sel.idx_sorted.cpu().numpy(),
+             order=sel.pick_order.cpu().numpy(), n_kept=sel.n_kept.cpu().numpy(), status=sel.status.cpu().numpy())
+    g["scores"] = akv.alpha_score(dev(ev.K), q, pos=dev(ev.pos), p_ref=pref).cpu().numpy()
+    check_all(ev, g, 0.5)
+
+
+def test_invalid_arguments_launch_nothing():
+    ev = synth.make_plain(1, 1, 1, 32, 128, 8, 0.5, dtype=synth.BF16, seed=26)
+    K, V, pos, q = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat)
+    before = akv.launch_count()
+    with pytest.raises(akv.AkvError) as e:
+        akv.alpha_compress_event(K, V, pos, q, 33)
+    assert e.value.code == 3
+    with pytest.raises(akv.AkvError) as e:
+        akv.alpha_compress_event(K, V, pos, q, 8, akv.Options(lam=-1.0))
+    assert e.value.code == 1
+    with pytest.raises(akv.AkvError) as e:
+        akv.alpha_compress_event(K.view(torch.int16)[..., 1:].view(torch.bfloat16) if False else K, V, pos, q, 8,
+                                 akv.Options(sig_mode=akv.SIG_FLAT))
+    assert e.value.code == 1
+    Kodd = torch.empty(32 * 128 + 8, dtype=torch.bfloat16, device="cuda")[4:4 + 32 * 128].view(1, 1, 1, 32, 128)
+    with pytest.raises(akv.AkvError) as e:
+        akv.alpha_score(Kodd, q)
+    assert e.value.code == 4
+    assert akv.launch_count() == before
+    assert np.array_equal(akv.to_host_bits(K), ev.K)

@@ -322,3 +322,14 @@ def test_replay_accepts_oracle_order_and_rejects_a_wrong_pick():
     dup = sel.order.copy()
     dup[3] = dup[1]
     assert not O.replay_pick_order(s, sig, 0.5, dup).ok
+
+
+def test_too_few_finite_scores_still_gives_distinct_indices():
+    s = np.array([np.nan, 1.0, np.inf, 0.5, -np.inf, np.nan])
+    sig = O.signatures_per_head(np.eye(6, dtype=np.float32))
+    for lam in (0.0, 0.5):
+        a = O.alpha_select(s, sig, 4, lam)
+        assert a.order[:2].tolist() == [1, 3]
+        assert len(set(a.order.tolist())) == 4 and a.order[2:].tolist() == [0, 2]
+        oc, _, _, st = CO.select(s, sig, 4, lam)
+        assert oc.tolist() == a.order.tolist() and st == O.STATUS_NONFINITE

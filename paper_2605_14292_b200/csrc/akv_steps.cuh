@@ -34,11 +34,22 @@ __device__ __forceinline__ void fold_query(const float* __restrict__ q, const Sc
     }
 }
 
-// cos and sin of 2*pi*frac where frac is the top 32 bits of a 0.64 fixed-point turn count
-__device__ __forceinline__ void sincos_turns(uint32_t top, float* sn, float* cs) {
-    // signed fraction of a turn in [-1/2, 1/2), as a multiple of pi in [-1, 1)
-    const float x = (float)(int32_t)top * 4.656612873077393e-10f;  // 2^-31
-    sincospif(x, sn, cs);
+// cos and sin of 2*pi*(top / 2^32): octant reduction on the fixed-point phase, then short polynomials
+// in y = (angle offset)/(pi/4) in [-1, 1) (least-squares fits at Chebyshev nodes, |error| < 1e-7).
+__device__ __forceinline__ void sincos_phase(uint32_t top, float& sn, float& cs) {
+    const uint32_t u = top + 0x20000000u;
+    const uint32_t quad = u >> 30;
+    const int t = (int)(u & 0x3FFFFFFFu) - 0x20000000;
+    const float y = (float)t * 1.862645149230957e-09f;  // 2^-29
+    const float z = y * y;
+    const float sp = y * fmaf(z, fmaf(z, fmaf(z, -3.587714997811334e-05f, 0.0024898717780787645f), -0.08074536717605851f),
+                              0.7853981525308736f);
+    const float cp = fmaf(z, fmaf(z, fmaf(z, -0.0003191315544232772f, 0.01585035496683941f), -0.308424473701413f), 1.0f);
+    const bool swap = quad & 1u;
+    const float c0 = swap ? sp : cp;
+    const float s0 = swap ? cp : sp;
+    cs = ((quad + 1u) & 2u) ? -c0 : c0;  // quadrants 1, 2
+    sn = (quad & 2u) ? -s0 : s0;         // quadrants 2, 3
 }
 
 // Score of one row, computed by the G lanes of a group; lane `lig` covers frequencies
@@ -61,7 +72,7 @@ __device__ __forceinline__ float score_row(const T* krow, bool valid, long long 
             if (rotate) {
                 const unsigned long long turns = (unsigned long long)dist * phi[f0 + u];
                 float sn, cs;
-                sincos_turns((uint32_t)(turns >> 32), &sn, &cs);
+                sincos_phase((uint32_t)(turns >> 32), sn, cs);
                 acc += fmaf(tr, cs, -ti * sn);
             } else {
                 acc += tr;

@@ -8,7 +8,7 @@
 #include <cstdio>
 #include <cstring>
 
-#include "akv_kernels.cuh"
+#include "akv_event_warp.cuh"
 
 using namespace akv;
 
@@ -265,7 +265,29 @@ static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStrea
     }
     return launched("select");
 }
+
+// Fast path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.
+static bool warp_path_ok(const EventArgs& a) {
+    return a.lay.dtype == AKV_BF16 && a.lay.d == kWD && a.lay.N <= 256 && a.flat_sig == nullptr;
+}
+template <bool FUSED>
+static akv_status_t launch_warp(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    akv_status_t s;
+    if (a.lay.N <= 192) {
+        const WarpSmem sp = plan_warp_smem(12, a.budget);
+        if ((s = set_smem(event_warp_kernel<12, FUSED>, sp.total)) != AKV_OK) return s;
+        event_warp_kernel<12, FUSED><<<E, kWThreads, sp.total, st>>>(a, h->tab);
+    } else {
+        const WarpSmem sp = plan_warp_smem(16, a.budget);
+        if ((s = set_smem(event_warp_kernel<16, FUSED>, sp.total)) != AKV_OK) return s;
+        event_warp_kernel<16, FUSED><<<E, kWThreads, sp.total, st>>>(a, h->tab);
+    }
+    return launched(FUSED ? "event_warp" : "select_warp");
+}
+
 static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    if (warp_path_ok(a) && a.V) return launch_warp<false>(h, a, st);
     return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st) : launch_select_t<float>(h, a, st);
 }
 
@@ -428,6 +450,7 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
     a.scores = scores; a.n_kept = n_kept; a.status = status;
 
+    if (warp_path_ok(a)) return launch_warp<true>(h, a, st);
     const int es = lay->dtype == AKV_BF16 ? 2 : 4;
     const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
     if ((int)res.total <= h->smem_optin) {

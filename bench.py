@@ -243,7 +243,7 @@ def run_gpu(args):
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
-                "kernel": "event_warp_kernel<12, fused>", "algorithmic_bytes_per_launch": bytes_per_launch}
+                "kernel": "event_tc_kernel<fused>", "algorithmic_bytes_per_launch": bytes_per_launch}
 
     # end to end: pinned host buffers -> device, the same C-ABI call, indices and kept counts back
     hK, hV, hP = (torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (K0, V0, P0))

@@ -1,0 +1,532 @@
+// Tensor-memory path for bf16, d = 128, per-head signatures, N <= 256: one CTA of four warps per
+// event, several CTAs resident per SM.
+//
+//   1. K rows arrive in shared memory by per-row bulk copies (cp.async.bulk + mbarrier) and are
+//      scored there (fused RoPE rotate-and-dot against the folded query statistic).
+//   2. Candidates are ranked by score (ties to the lower slot). Only candidates with
+//        s_i >= s_(b) - lambda * (1 + slack)
+//      can ever be an argmax of Eq. 2 (the running maximum m never exceeds 1, so every still
+//      unchosen member of the top-b scores beats them): that pool of P rows, in rank order, is
+//      the only part of V that is read.
+//   3. The pool's V rows are laid out as a K-major, 128-byte-swizzled operand tile and ONE
+//      tcgen05.mma sequence writes the pool's cosine matrix (raw dot products, fp32) into tensor
+//      memory: row rho lives in TMEM lane rho, column c holds <V_rho, V_c>.
+//   4. Algorithm 1 runs with one candidate per thread (two when P > 128): a = s - lambda m in
+//      registers, warp redux + one shared-memory exchange per pick for the argmax, then every
+//      thread pulls its own entry of the picked column from tensor memory (tcgen05.ld).
+//   5. Kept rows are written back in place: V from the tile, K and positions re-read (L2) and
+//      staged on chip before the first store.
+#pragma once
+#include "akv_kernels.cuh"
+
+namespace akv {
+
+constexpr int kTcThreads = 128;
+constexpr int kTcD = 128;        // head dimension of this path
+constexpr int kTcMaxN = 256;     // most candidates per event
+constexpr int kTcCols = 128;     // cosine-matrix columns kept in tensor memory per block of 128 rows
+constexpr int kWaitPolls = 1 << 22;
+
+struct TcSmem {
+    unsigned tile, s, key, spos, byrank, rankof, taken, order, gain, idx, slot, misc, total;
+    int tile_rows;
+};
+// Layout after the 1024-byte aligned base. `key` (ranking) and `r` (reciprocal norms) share storage.
+__host__ __device__ inline TcSmem plan_tc_smem(int N, int budget) {
+    TcSmem p;
+    p.tile_rows = ((N + 7) & ~7) < 128 ? 128 : ((N + 7) & ~7);
+    const unsigned np = (unsigned)((N + 3) & ~3);
+    unsigned o = 0;
+    p.tile = o;   o += (unsigned)p.tile_rows * 256u;
+    p.s = o;      o += align16(np * 4);
+    p.key = o;    o += align16(np * 4);
+    p.spos = o;   o += align16(np * 4);
+    p.byrank = o; o += align16(np * 2);
+    p.rankof = o; o += align16(np * 2);
+    p.taken = o;  o += align16(np);
+    p.order = o;  o += align16((unsigned)budget * 4);
+    p.gain = o;   o += align16((unsigned)budget * 4);
+    p.idx = o;    o += align16((unsigned)budget * 4);
+    p.slot = o;   o += 64;   // 2 x 4 keys of 8 bytes
+    p.misc = o;   o += 64;   // mbarriers (2 x 8), tmem base, s_(b), block-max scratch
+    p.total = o + 1024;      // room to align the base to 1024 bytes
+    return p;
+}
+
+// ---- PTX wrappers --------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after a fixed number of polls instead of spinning for ever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (int it = 0; it < kWaitPolls; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t holder, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulation; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// One fp32 per thread: TMEM lane = (warp % 4) * 32 + lane, column given by the address.
+__device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
+    uint32_t v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(taddr) : "memory");
+    return __uint_as_float(v);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart (the tile base is 1024-byte aligned).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+    d |= (uint64_t)(1024u >> 4) << 32;         // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
+__host__ __device__ inline uint32_t umma_idesc_bf16(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// byte offset inside the operand tile of 16-byte chunk c (0..15) of pool row rho
+__device__ __forceinline__ uint32_t tile_chunk(int rho, int c, uint32_t half_bytes) {
+    return (uint32_t)(c >> 3) * half_bytes + (uint32_t)rho * 128u + (uint32_t)(((c & 7) ^ (rho & 7)) << 4);
+}
+
+// 64-bit argmax key: score key | 0xFFFF - original slot | pool row. Larger wins; equal values go to
+// the lower original slot.
+__device__ __forceinline__ uint32_t key_low(int orig, int rho) { return ((0xFFFFu - (uint32_t)orig) << 16) | (uint32_t)rho; }
+
+// ---- the kernel ------------------------------------------------------------------------------------
+// FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
+// nothing is rewritten).
+template <bool FUSED>
+__global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int n = event_n(a, id.b);
+    const int N = lay.N;
+    const int picks = min(a.budget, n);
+    const TcSmem sp = plan_tc_smem(N, a.budget);
+    unsigned char* tile = smem + sp.tile;
+    float* s = reinterpret_cast<float*>(smem + sp.s);
+    uint32_t* key = reinterpret_cast<uint32_t*>(smem + sp.key);
+    float* r = reinterpret_cast<float*>(smem + sp.key);  // reuses the ranking keys' storage
+    int* spos = reinterpret_cast<int*>(smem + sp.spos);
+    unsigned short* byrank = reinterpret_cast<unsigned short*>(smem + sp.byrank);
+    unsigned short* rankof = reinterpret_cast<unsigned short*>(smem + sp.rankof);
+    unsigned char* taken = smem + sp.taken;
+    int* order = reinterpret_cast<int*>(smem + sp.order);
+    float* gain = reinterpret_cast<float*>(smem + sp.gain);
+    int* idx = reinterpret_cast<int*>(smem + sp.idx);
+    uint2* slot = reinterpret_cast<uint2*>(smem + sp.slot);
+    const uint32_t barK = smem_u32(smem + sp.misc);
+    const uint32_t barM = barK + 8;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 16);
+    float* sb_holder = reinterpret_cast<float*>(smem + sp.misc + 20);
+    int* redi = reinterpret_cast<int*>(smem + sp.misc + 32);
+    const uint32_t tile_u32 = smem_u32(tile);
+    const uint32_t half_bytes = (uint32_t)sp.tile_rows * 128u;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(a.K);
+    __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
+    const bool similarity = a.greedy != 0;
+    const int np4 = (N + 3) & ~3;
+
+    if (tid == 0) {
+        mbar_init(barK, 1);
+        mbar_init(barM, 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    // ---- scores ---------------------------------------------------------------------------------
+    int bad = 0;
+    int timeout = 0;
+    if (FUSED) {
+        if (tid == 0) mbar_expect_tx(barK, (uint32_t)n * 256u);
+        for (int row = tid; row < n; row += kTcThreads)
+            bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row), 256u, barK);
+        const int* gpos = event_pos(a.pos, id);
+        const bool rotate = gpos != nullptr;
+        int pmax = INT_MIN;
+        for (int j = tid; j < n; j += kTcThreads) {
+            const int p = rotate ? gpos[j] : 0;
+            spos[j] = p;
+            pmax = max(pmax, p);
+        }
+        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
+        const int grp = lane >> 3, f0 = (lane & 7) * 8;
+        const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
+        const float inv = rsqrtf((float)kTcD);
+        float2 g[8];
+        uint32_t phi_lo[8], phi_hi[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float qr = q[f0 + u] * inv, qi = q[f0 + u + 64] * inv;
+            const float2 c = tab.cw[f0 + u];
+            g[u] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+            phi_lo[u] = (uint32_t)tab.phi[f0 + u];
+            phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
+        }
+        long long pref = 0;
+        if (rotate) {
+            if (a.p_ref) {
+                pref = a.p_ref[id.b];
+                __syncthreads();
+            } else {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
+                if (lane == 0) redi[warp] = pmax;
+                __syncthreads();
+                pref = (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
+            }
+        } else {
+            __syncthreads();
+        }
+        timeout = !mbar_wait_bounded(barK, 0);
+        if (!timeout) {
+            for (int j0 = 4 * warp; j0 < n; j0 += 4 * (kTcThreads / 32)) {
+                const int j = j0 + grp;
+                float acc = 0.f;
+                if (j < n) {
+                    const uint4 wr = *reinterpret_cast<const uint4*>(tile + j * 256 + (lane & 7) * 16);
+                    const uint4 wi = *reinterpret_cast<const uint4*>(tile + j * 256 + 128 + (lane & 7) * 16);
+                    const float kre[8] = {bf16lo(wr.x), bf16hi(wr.x), bf16lo(wr.y), bf16hi(wr.y),
+                                          bf16lo(wr.z), bf16hi(wr.z), bf16lo(wr.w), bf16hi(wr.w)};
+                    const float kim[8] = {bf16lo(wi.x), bf16hi(wi.x), bf16lo(wi.y), bf16hi(wi.y),
+                                          bf16lo(wi.z), bf16hi(wi.z), bf16lo(wi.w), bf16hi(wi.w)};
+                    const long long dist = pref - (long long)spos[j];
+                    const uint32_t dlo = (uint32_t)dist, dhi = (uint32_t)((unsigned long long)dist >> 32);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const float tr = fmaf(g[u].x, kre[u], g[u].y * kim[u]);
+                        const float ti = fmaf(g[u].y, kre[u], -g[u].x * kim[u]);
+                        if (rotate) {
+                            // bits 32..63 of dist * phi (mod 2^64)
+                            const uint32_t top = __umulhi(dlo, phi_lo[u]) + dlo * phi_hi[u] + dhi * phi_lo[u];
+                            float sn, cs;
+                            sincos_phase(top, sn, cs);
+                            acc += fmaf(tr, cs, -ti * sn);
+                        } else {
+                            acc += tr;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+                if (j < n && (lane & 7) == 0) {
+                    if (a.scores) a.scores[(long long)id.e * N + j] = acc;
+                    const bool fin = isfinite(acc);
+                    bad |= !fin;
+                    const float sj = fin ? acc : -INFINITY;
+                    s[j] = sj;
+                    key[j] = orderable(sj);
+                }
+            }
+        }
+    } else {
+        for (int j = tid; j < n; j += kTcThreads) {
+            const float sc = a.scores[(long long)id.e * N + j];
+            const bool fin = isfinite(sc);
+            bad |= !fin;
+            const float sj = fin ? sc : -INFINITY;
+            s[j] = sj;
+            key[j] = orderable(sj);
+        }
+    }
+    for (int j = n + tid; j < np4; j += kTcThreads) key[j] = 0u;  // below every real key
+    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
+    timeout = __syncthreads_or(timeout);
+    if (timeout) {
+        if (tid == 0 && a.status) a.status[id.e] = 3;
+        mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
+        return;
+    }
+    bad = __syncthreads_or(bad);
+
+    // ---- rank by score (ties to the lower slot) and the pool that can ever be picked ----------------
+    int cand[2], rank[2];
+    float sc[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int c = tid + u * kTcThreads;
+        cand[u] = c;
+        rank[u] = 0;
+        sc[u] = 0.f;
+        if (c < n) {
+            const uint32_t kc = key[c];
+            sc[u] = s[c];
+            int cnt = 0;
+            const uint4* k4 = reinterpret_cast<const uint4*>(key);
+            // slots below c win ties: count keys >= kc there, keys > kc at and above c
+            for (int i4 = 0; i4 < np4 / 4; ++i4) {
+                const uint4 kk = k4[i4];
+                const int i = 4 * i4;
+                cnt += (kk.x > kc - (uint32_t)(i < c)) + (kk.y > kc - (uint32_t)(i + 1 < c)) +
+                       (kk.z > kc - (uint32_t)(i + 2 < c)) + (kk.w > kc - (uint32_t)(i + 3 < c));
+            }
+            rank[u] = cnt;
+        }
+    }
+    __syncthreads();  // every key has been read: its storage becomes r below
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        if (cand[u] < n) {
+            byrank[rank[u]] = (unsigned short)cand[u];
+            rankof[cand[u]] = (unsigned short)rank[u];
+            if (rank[u] == picks - 1) *sb_holder = sc[u];
+        }
+    }
+    __syncthreads();
+    int P = picks;
+    if (similarity && picks > 0) {
+        if (a.no_prune) {
+            P = n;
+        } else {
+            const float sb = *sb_holder;
+            const float thr = fmaf(-1.001f, a.lam, sb) - 1e-6f * fabsf(sb);  // -inf keeps everyone
+            const int in0 = cand[0] < n && !(sc[0] < thr);
+            const int in1 = cand[1] < n && !(sc[1] < thr);
+            P = __syncthreads_count(in0) + __syncthreads_count(in1);
+        }
+    }
+    const bool two = P > 128;                      // second block of 128 rows ends at the pool's last row
+    const int base2 = two ? ((P + 7) & ~7) - 128 : 0;
+    const int ncols = min((P + 15) & ~15, kTcCols);  // columns of the cosine matrix held in tensor memory
+    const uint32_t tcols = two ? 256u : (ncols <= 32 ? 32u : (ncols <= 64 ? 64u : 128u));
+    const bool use_tc = similarity && picks > 1;
+
+    // ---- V rows of the pool, in rank order, as the swizzled operand tile ---------------------------
+    const int vrows = (similarity || FUSED) ? P : 0;
+    for (int x = tid; x < vrows * 16; x += kTcThreads) {
+        const int rho = x >> 4, c = x & 15;
+        const int j = byrank[rho];
+        cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + row_offset(lay, id.b, id.l, id.h, j) + c * 8);
+    }
+    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), tcols);
+    cp_async_wait_all();
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = use_tc ? *tmem_holder : 0u;
+
+    if (use_tc && tid == 0) {
+        const uint32_t idesc = umma_idesc_bf16(128, ncols);
+#pragma unroll 1
+        for (int blk = 0; blk < (two ? 2 : 1); ++blk) {
+            const uint32_t arow = tile_u32 + (uint32_t)(blk ? base2 : 0) * 128u;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
+                umma_bf16(tbase + (uint32_t)blk * kTcCols, umma_desc_sw128(arow + koff), umma_desc_sw128(tile_u32 + koff),
+                          idesc, kk > 0 ? 1u : 0u);
+            }
+        }
+        umma_commit(barM);
+    }
+
+    // ---- reciprocal norms of the pool rows (Eq. 1), while the tensor core works ----------------------
+    int rho[2] = {tid, base2 + tid};
+    bool mine[2] = {tid < P, two && base2 + tid >= 128 && base2 + tid < P};
+    float sv[2] = {0.f, 0.f}, lr[2] = {0.f, 0.f}, M[2] = {0.f, 0.f};
+    uint32_t klow[2] = {0u, 0u};
+    if (!similarity) mine[0] = mine[1] = false;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        if (mine[u]) {
+            const int j = byrank[rho[u]];
+            sv[u] = s[j];
+            klow[u] = key_low(j, rho[u]);
+            if (similarity) {
+                float ss = 0.f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float x[8];
+                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho[u], c, half_bytes)), x);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
+                }
+                const float rr = 1.f / (sqrtf(ss) + a.eps);
+                r[rho[u]] = rr;
+                lr[u] = a.lam * rr;
+            }
+        }
+    }
+    if (use_tc) timeout = !mbar_wait_bounded(barM, 0);
+    tc_fence_after();
+    timeout = __syncthreads_or(timeout);
+    if (timeout) {
+        if (tid == 0 && a.status) a.status[id.e] = 3;
+        if (use_tc && warp == 0) tmem_dealloc(tbase, tcols);
+        return;
+    }
+
+    // ---- Algorithm 1 ----------------------------------------------------------------------------------
+    const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);
+    if (!similarity) {
+        // lambda = 0: the first `picks` ranks are the answer, in pick order
+        for (int t = tid; t < picks; t += kTcThreads) {
+            const int j = byrank[t];
+            order[t] = j;
+            gain[t] = s[j];
+            taken[j] = 1;
+        }
+    }
+    for (int t = 0; similarity && t < picks; ++t) {
+        // a = s - lambda m (a[S] = -inf: chosen candidates no longer compete); i = argmax a
+        uint32_t khi = 0u, klo = 0u;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (mine[u]) {
+                const uint32_t k = orderable(fmaf(-lr[u], M[u], sv[u]));
+                if (k > khi || (k == khi && klow[u] > klo)) { khi = k; klo = klow[u]; }
+            }
+        }
+        const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, khi);
+        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, khi == whi ? klo : 0u);
+        uint2* sl = slot + (t & 1) * 4;
+        if (lane == 0) sl[warp] = make_uint2(whi, wlo);
+        __syncthreads();
+        uint2 best = sl[0];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+            const uint2 o = sl[w];
+            if (o.x > best.x || (o.x == best.x && o.y > best.y)) best = o;
+        }
+        const int irho = (int)(best.y & 0xFFFFu);
+        const int iorig = (int)(0xFFFFu - (best.y >> 16));
+        if (tid == 0) {
+            order[t] = iorig;
+            gain[t] = from_orderable(best.x);
+            taken[iorig] = 1;
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (mine[u] && rho[u] == irho) mine[u] = false;
+        if (t + 1 == picks) continue;
+        // m <- max(m, Sims[i, :]): every thread reads its own rows' entries of column i
+        const float ri = r[irho];
+        float d0, d1 = 0.f;
+        if (irho < ncols) {
+            d0 = tmem_ld1(tlane + (uint32_t)irho);
+            if (two) d1 = tmem_ld1(tlane + (uint32_t)(kTcCols + irho));
+            tmem_ld_wait();
+        } else {
+            // the picked row lies outside the stored columns: plain dot products from the tile
+            float acc[2] = {0.f, 0.f};
+#pragma unroll 4
+            for (int c = 0; c < 16; ++c) {
+                float vi[8];
+                load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(irho, c, half_bytes)), vi);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if (mine[u]) {
+                        float vj[8];
+                        load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho[u], c, half_bytes)), vj);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[u] = fmaf(vi[e], vj[e], acc[u]);
+                    }
+                }
+            }
+            d0 = acc[0];
+            d1 = acc[1];
+        }
+        M[0] = fmaxf(M[0], ri * d0);
+        M[1] = fmaxf(M[1], ri * d1);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (use_tc && warp == 0) tmem_dealloc(tbase, tcols);
+
+    // ---- sort(S) and outputs -------------------------------------------------------------------------
+    ordered_indices(n, a.budget, taken, idx);
+    __syncthreads();
+    const long long ob = (long long)id.e * a.budget;
+    for (int t = tid; t < a.budget; t += kTcThreads) {
+        a.idx_sorted[ob + t] = idx[t];
+        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
+        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
+    }
+    if (tid == 0) {
+        if (a.n_kept) a.n_kept[id.e] = picks;
+        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+    }
+    if (!FUSED) return;
+
+    // ---- compaction in place: V from the tile; K and positions staged on chip before any store -----
+    for (int x = tid; x < picks * 16; x += kTcThreads) {
+        const int rr = x >> 4, c = x & 15;
+        copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
+               tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
+    }
+    int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
+    __syncthreads();  // the V tile is free from here on
+    __nv_bfloat16* Kw = reinterpret_cast<__nv_bfloat16*>(a.K);
+    for (int x = tid; x < picks * 16; x += kTcThreads) {
+        const int rr = x >> 4, c = x & 15;
+        copy16(tile + rr * 256 + c * 16, reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[rr])) + c * 16);
+    }
+    __syncthreads();
+    for (int x = tid; x < picks * 16; x += kTcThreads) {
+        const int rr = x >> 4, c = x & 15;
+        copy16(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16, tile + rr * 256 + c * 16);
+    }
+    if (wpos)
+        for (int t = tid; t < picks; t += kTcThreads) wpos[t] = spos[idx[t]];
+}
+
+}  // namespace akv

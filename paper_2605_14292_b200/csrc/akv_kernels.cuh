@@ -16,6 +16,7 @@ struct EventArgs {
     int budget;
     float lam, eps;
     int greedy;             // 1: run the loop with similarity updates; 0: top-k
+    int no_prune;           // 1: keep every candidate in the pool the loop runs over
     int* idx_sorted;
     int* pick_order;
     float* pick_gain;

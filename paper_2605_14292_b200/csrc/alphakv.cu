@@ -8,7 +8,7 @@
 #include <cstdio>
 #include <cstring>
 
-#include "akv_event_warp.cuh"
+#include "akv_event_tc.cuh"
 
 using namespace akv;
 
@@ -266,28 +266,25 @@ static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStrea
     return launched("select");
 }
 
-// Fast path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.
-static bool warp_path_ok(const EventArgs& a) {
-    return a.lay.dtype == AKV_BF16 && a.lay.d == kWD && a.lay.N <= 256 && a.flat_sig == nullptr;
+// Tensor-memory path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.
+static bool tc_path_ok(const EventArgs& a) {
+    return a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.flat_sig == nullptr;
 }
 template <bool FUSED>
-static akv_status_t launch_warp(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+static akv_status_t launch_tc(akv_handle* h, const EventArgs& a, cudaStream_t st) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
+    const TcSmem sp = plan_tc_smem(a.lay.N, a.budget);
+    if ((int)sp.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "budget %d needs too much shared memory", a.budget);
     akv_status_t s;
-    if (a.lay.N <= 192) {
-        const WarpSmem sp = plan_warp_smem(12, a.budget);
-        if ((s = set_smem(event_warp_kernel<12, FUSED>, sp.total)) != AKV_OK) return s;
-        event_warp_kernel<12, FUSED><<<E, kWThreads, sp.total, st>>>(a, h->tab);
-    } else {
-        const WarpSmem sp = plan_warp_smem(16, a.budget);
-        if ((s = set_smem(event_warp_kernel<16, FUSED>, sp.total)) != AKV_OK) return s;
-        event_warp_kernel<16, FUSED><<<E, kWThreads, sp.total, st>>>(a, h->tab);
-    }
-    return launched(FUSED ? "event_warp" : "select_warp");
+    if ((s = set_smem(event_tc_kernel<FUSED>, sp.total)) != AKV_OK) return s;
+    CUDA_TRY(cudaFuncSetAttribute(event_tc_kernel<FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                  (int)cudaSharedmemCarveoutMaxShared));
+    event_tc_kernel<FUSED><<<E, kTcThreads, sp.total, st>>>(a, h->tab);
+    return launched(FUSED ? "event_tc" : "select_tc");
 }
 
 static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st) {
-    if (warp_path_ok(a) && a.V) return launch_warp<false>(h, a, st);
+    if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st);
     return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st) : launch_select_t<float>(h, a, st);
 }
 
@@ -342,6 +339,7 @@ static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, con
     a.lam = opt->lambda;
     a.eps = opt->eps;
     a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
+    a.no_prune = (opt->flags & AKV_FLAG_NO_PRUNE) ? 1 : 0;
     if (opt->sig_mode == AKV_SIG_FLAT) {
         if (!flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat signature mode needs flat_sig");
         if (!aligned16(flat_sig)) return fail(AKV_ERR_ALIGNMENT, "flat_sig is not 16-byte aligned");
@@ -450,7 +448,7 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
     a.scores = scores; a.n_kept = n_kept; a.status = status;
 
-    if (warp_path_ok(a)) return launch_warp<true>(h, a, st);
+    if (tc_path_ok(a)) return launch_tc<true>(h, a, st);
     const int es = lay->dtype == AKV_BF16 ? 2 : 4;
     const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
     if ((int)res.total <= h->smem_optin) {

@@ -185,12 +185,20 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     const bool similarity = a.greedy != 0;
     const int np4 = (N + 3) & ~3;
 
+    // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
+    // next CTA of this kernel only after that, so a late allocation would serialise the CTAs.
+    const uint32_t tcols = (uint32_t)a.tmem_cols;
+    const bool use_tc = similarity && tcols != 0u;
     if (tid == 0) {
         mbar_init(barK, 1);
         mbar_init(barM, 1);
         mbar_init_fence();
     }
+    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), tcols);
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = use_tc ? *tmem_holder : 0u;
 
     // ---- scores ---------------------------------------------------------------------------------
     int bad = 0;
@@ -293,6 +301,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
         mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
+        if (use_tc && warp == 0) tmem_dealloc(tbase, tcols);
         return;
     }
     bad = __syncthreads_or(bad);
@@ -309,15 +318,19 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         if (c < n) {
             const uint32_t kc = key[c];
             sc[u] = s[c];
+            // slots below c win ties: count keys >= kc there (k > kc - 1) and keys > kc from c on;
+            // the group of four that holds c is counted with > kc and corrected for equal keys below c
             int cnt = 0;
             const uint4* k4 = reinterpret_cast<const uint4*>(key);
-            // slots below c win ties: count keys >= kc there, keys > kc at and above c
+            const int g = c >> 2;
             for (int i4 = 0; i4 < np4 / 4; ++i4) {
                 const uint4 kk = k4[i4];
-                const int i = 4 * i4;
-                cnt += (kk.x > kc - (uint32_t)(i < c)) + (kk.y > kc - (uint32_t)(i + 1 < c)) +
-                       (kk.z > kc - (uint32_t)(i + 2 < c)) + (kk.w > kc - (uint32_t)(i + 3 < c));
+                const uint32_t thr = i4 < g ? kc - 1u : kc;
+                cnt += (kk.x > thr) + (kk.y > thr) + (kk.z > thr) + (kk.w > thr);
             }
+            const uint4 kg = k4[g];
+            const int e = c & 3;
+            cnt += (e > 0 && kg.x == kc) + (e > 1 && kg.y == kc) + (e > 2 && kg.z == kc);
             rank[u] = cnt;
         }
     }
@@ -345,9 +358,10 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     }
     const bool two = P > 128;                      // second block of 128 rows ends at the pool's last row
     const int base2 = two ? ((P + 7) & ~7) - 128 : 0;
-    const int ncols = min((P + 15) & ~15, kTcCols);  // columns of the cosine matrix held in tensor memory
-    const uint32_t tcols = two ? 256u : (ncols <= 32 ? 32u : (ncols <= 64 ? 64u : 128u));
-    const bool use_tc = similarity && picks > 1;
+    // columns of the cosine matrix held in tensor memory (per block of 128 rows); picks of a later
+    // rank take the plain dot-product route below
+    const int cstride = two ? (int)(tcols >> 1) : (int)tcols;
+    const int ncols = min((P + 15) & ~15, min(cstride, 128));
 
     // ---- V rows of the pool, in rank order, as the swizzled operand tile ---------------------------
     const int vrows = (similarity || FUSED) ? P : 0;
@@ -356,15 +370,13 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         const int j = byrank[rho];
         cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + row_offset(lay, id.b, id.l, id.h, j) + c * 8);
     }
-    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), tcols);
     cp_async_wait_all();
     fence_proxy_async();
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tbase = use_tc ? *tmem_holder : 0u;
 
-    if (use_tc && tid == 0) {
+    const bool do_mma = use_tc && picks > 1;
+    if (do_mma && tid == 0) {
+        tc_fence_after();
         const uint32_t idesc = umma_idesc_bf16(128, ncols);
 #pragma unroll 1
         for (int blk = 0; blk < (two ? 2 : 1); ++blk) {
@@ -372,7 +384,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
-                umma_bf16(tbase + (uint32_t)blk * kTcCols, umma_desc_sw128(arow + koff), umma_desc_sw128(tile_u32 + koff),
+                umma_bf16(tbase + (uint32_t)(blk * cstride), umma_desc_sw128(arow + koff), umma_desc_sw128(tile_u32 + koff),
                           idesc, kk > 0 ? 1u : 0u);
             }
         }
@@ -406,7 +418,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
             }
         }
     }
-    if (use_tc) timeout = !mbar_wait_bounded(barM, 0);
+    if (do_mma) timeout = !mbar_wait_bounded(barM, 0);
     tc_fence_after();
     timeout = __syncthreads_or(timeout);
     if (timeout) {
@@ -426,71 +438,105 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
             taken[j] = 1;
         }
     }
-    for (int t = 0; similarity && t < picks; ++t) {
-        // a = s - lambda m (a[S] = -inf: chosen candidates no longer compete); i = argmax a
-        uint32_t khi = 0u, klo = 0u;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            if (mine[u]) {
-                const uint32_t k = orderable(fmaf(-lr[u], M[u], sv[u]));
-                if (k > khi || (k == khi && klow[u] > klo)) { khi = k; klo = klow[u]; }
-            }
-        }
-        const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, khi);
-        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, khi == whi ? klo : 0u);
-        uint2* sl = slot + (t & 1) * 4;
-        if (lane == 0) sl[warp] = make_uint2(whi, wlo);
-        __syncthreads();
-        uint2 best = sl[0];
-#pragma unroll
-        for (int w = 1; w < 4; ++w) {
-            const uint2 o = sl[w];
-            if (o.x > best.x || (o.x == best.x && o.y > best.y)) best = o;
-        }
-        const int irho = (int)(best.y & 0xFFFFu);
-        const int iorig = (int)(0xFFFFu - (best.y >> 16));
-        if (tid == 0) {
-            order[t] = iorig;
-            gain[t] = from_orderable(best.x);
-            taken[iorig] = 1;
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            if (mine[u] && rho[u] == irho) mine[u] = false;
-        if (t + 1 == picks) continue;
-        // m <- max(m, Sims[i, :]): every thread reads its own rows' entries of column i
-        const float ri = r[irho];
-        float d0, d1 = 0.f;
-        if (irho < ncols) {
-            d0 = tmem_ld1(tlane + (uint32_t)irho);
-            if (two) d1 = tmem_ld1(tlane + (uint32_t)(kTcCols + irho));
+    // The winning key of every pick is parked in order[] (low word) and gain[] (high word) and
+    // decoded after the loop.
+    uint32_t* park_lo = reinterpret_cast<uint32_t*>(order);
+    uint32_t* park_hi = reinterpret_cast<uint32_t*>(gain);
+    if (similarity && !two) {
+        // one candidate per thread
+        const int myrho = tid;
+        bool live = mine[0];
+        const float s0 = sv[0], lr0 = lr[0];
+        const uint32_t kl0 = klow[0];
+        float M0 = 0.f;
+        for (int t = 0; t < picks; ++t) {
+            // a = s - lambda m (a[S] = -inf: chosen candidates no longer compete); i = argmax a
+            const uint32_t khi = live ? orderable(fmaf(-lr0, M0, s0)) : 0u;
+            const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, khi);
+            const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, khi == whi ? kl0 : 0u);
+            uint2* sl = slot + (t & 1) * 4;
+            if (lane == 0) sl[warp] = make_uint2(whi, wlo);
+            __syncthreads();
+            const uint2 mk = sl[lane & 3];
+            const uint32_t bhi = __reduce_max_sync(0xFFFFFFFFu, mk.x);
+            const uint32_t blo = __reduce_max_sync(0xFFFFFFFFu, mk.x == bhi ? mk.y : 0u);
+            const int irho = (int)(blo & 0xFFFFu);
+            if (tid == 0) { park_hi[t] = bhi; park_lo[t] = blo; }
+            live = live && myrho != irho;
+            if (t + 1 == picks) break;
+            // m <- max(m, Sims[i, :]): every thread reads its own row's entry of column i
+            const float ri = r[irho];
+            const float d0 = tmem_ld1(tlane + (uint32_t)irho);
             tmem_ld_wait();
-        } else {
-            // the picked row lies outside the stored columns: plain dot products from the tile
-            float acc[2] = {0.f, 0.f};
-#pragma unroll 4
-            for (int c = 0; c < 16; ++c) {
-                float vi[8];
-                load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(irho, c, half_bytes)), vi);
+            M0 = fmaxf(M0, ri * d0);
+        }
+    } else if (similarity) {
+        // two candidates per thread; picks beyond the stored columns use plain dot products
+        for (int t = 0; t < picks; ++t) {
+            uint32_t khi = 0u, klo = 0u;
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    if (mine[u]) {
-                        float vj[8];
-                        load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho[u], c, half_bytes)), vj);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[u] = fmaf(vi[e], vj[e], acc[u]);
-                    }
+            for (int u = 0; u < 2; ++u) {
+                if (mine[u]) {
+                    const uint32_t k = orderable(fmaf(-lr[u], M[u], sv[u]));
+                    if (k > khi || (k == khi && klow[u] > klo)) { khi = k; klo = klow[u]; }
                 }
             }
-            d0 = acc[0];
-            d1 = acc[1];
+            const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, khi);
+            const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, khi == whi ? klo : 0u);
+            uint2* sl = slot + (t & 1) * 4;
+            if (lane == 0) sl[warp] = make_uint2(whi, wlo);
+            __syncthreads();
+            const uint2 mk = sl[lane & 3];
+            const uint32_t bhi = __reduce_max_sync(0xFFFFFFFFu, mk.x);
+            const uint32_t blo = __reduce_max_sync(0xFFFFFFFFu, mk.x == bhi ? mk.y : 0u);
+            const int irho = (int)(blo & 0xFFFFu);
+            if (tid == 0) { park_hi[t] = bhi; park_lo[t] = blo; }
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                if (mine[u] && rho[u] == irho) mine[u] = false;
+            if (t + 1 == picks) break;
+            const float ri = r[irho];
+            float d0, d1;
+            if (irho < ncols) {
+                d0 = tmem_ld1(tlane + (uint32_t)irho);
+                d1 = tmem_ld1(tlane + (uint32_t)(cstride + irho));
+                tmem_ld_wait();
+            } else {
+                float acc[2] = {0.f, 0.f};
+#pragma unroll 4
+                for (int c = 0; c < 16; ++c) {
+                    float vi[8];
+                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(irho, c, half_bytes)), vi);
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        if (mine[u]) {
+                            float vj[8];
+                            load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho[u], c, half_bytes)), vj);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[u] = fmaf(vi[e], vj[e], acc[u]);
+                        }
+                    }
+                }
+                d0 = acc[0];
+                d1 = acc[1];
+            }
+            M[0] = fmaxf(M[0], ri * d0);
+            M[1] = fmaxf(M[1], ri * d1);
         }
-        M[0] = fmaxf(M[0], ri * d0);
-        M[1] = fmaxf(M[1], ri * d1);
     }
     tc_fence_before();
     __syncthreads();
     if (use_tc && warp == 0) tmem_dealloc(tbase, tcols);
+    if (similarity) {
+        for (int t = tid; t < picks; t += kTcThreads) {
+            const uint32_t hi = park_hi[t], lo = park_lo[t];
+            const int j = (int)(0xFFFFu - (lo >> 16));
+            order[t] = j;
+            gain[t] = from_orderable(hi);
+            taken[j] = 1;
+        }
+        __syncthreads();
+    }
 
     // ---- sort(S) and outputs -------------------------------------------------------------------------
     ordered_indices(n, a.budget, taken, idx);
@@ -507,23 +553,50 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     }
     if (!FUSED) return;
 
-    // ---- compaction in place: V from the tile; K and positions staged on chip before any store -----
-    for (int x = tid; x < picks * 16; x += kTcThreads) {
-        const int rr = x >> 4, c = x & 15;
-        copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
-               tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
-    }
+    // ---- compaction in place ----------------------------------------------------------------------
+    // Every kept K row and position is on chip (registers for up to 64 rows, else the tile) before
+    // the first store: a destination slot can be another kept row's source.
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
-    __syncthreads();  // the V tile is free from here on
     __nv_bfloat16* Kw = reinterpret_cast<__nv_bfloat16*>(a.K);
-    for (int x = tid; x < picks * 16; x += kTcThreads) {
-        const int rr = x >> 4, c = x & 15;
-        copy16(tile + rr * 256 + c * 16, reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[rr])) + c * 16);
-    }
-    __syncthreads();
-    for (int x = tid; x < picks * 16; x += kTcThreads) {
-        const int rr = x >> 4, c = x & 15;
-        copy16(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16, tile + rr * 256 + c * 16);
+    if (picks <= 64) {
+        uint4 kreg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int x = tid + i * kTcThreads;
+            if (x < picks * 16)
+                kreg[i] = *reinterpret_cast<const uint4*>(
+                    reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[x >> 4])) + (x & 15) * 16);
+        }
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const int rr = x >> 4, c = x & 15;
+            copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
+                   tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
+        }
+        __syncthreads();  // every K load above has been performed
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int x = tid + i * kTcThreads;
+            if (x < picks * 16)
+                *reinterpret_cast<uint4*>(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, x >> 4)) + (x & 15) * 16) =
+                    kreg[i];
+        }
+    } else {
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const int rr = x >> 4, c = x & 15;
+            copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
+                   tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
+        }
+        __syncthreads();  // the V tile is free from here on
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const int rr = x >> 4, c = x & 15;
+            copy16(tile + rr * 256 + c * 16,
+                   reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[rr])) + c * 16);
+        }
+        __syncthreads();
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const int rr = x >> 4, c = x & 15;
+            copy16(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16, tile + rr * 256 + c * 16);
+        }
     }
     if (wpos)
         for (int t = tid; t < picks; t += kTcThreads) wpos[t] = spos[idx[t]];

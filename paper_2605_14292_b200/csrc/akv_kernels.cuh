@@ -17,6 +17,7 @@ struct EventArgs {
     float lam, eps;
     int greedy;             // 1: run the loop with similarity updates; 0: top-k
     int no_prune;           // 1: keep every candidate in the pool the loop runs over
+    int tmem_cols;          // tensor-memory columns the tensor-memory kernel claims per CTA (0: none)
     int* idx_sorted;
     int* pick_order;
     float* pick_gain;

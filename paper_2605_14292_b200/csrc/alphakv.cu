@@ -271,9 +271,13 @@ static bool tc_path_ok(const EventArgs& a) {
     return a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.flat_sig == nullptr;
 }
 template <bool FUSED>
-static akv_status_t launch_tc(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t st) {
+    EventArgs a = a0;
     const int E = a.lay.B * a.lay.L * a.lay.H;
     const TcSmem sp = plan_tc_smem(a.lay.N, a.budget);
+    // 512 columns per SM are shared by the resident CTAs. A pool of more than 128 rows needs two
+    // row blocks; with a small budget 64 columns per block hold nearly every pick.
+    a.tmem_cols = !a.greedy ? 0 : (a.lay.N <= 128 || a.budget <= 64) ? 128 : 256;
     if ((int)sp.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "budget %d needs too much shared memory", a.budget);
     akv_status_t s;
     if ((s = set_smem(event_tc_kernel<FUSED>, sp.total)) != AKV_OK) return s;

@@ -146,6 +146,31 @@ __device__ __forceinline__ uint32_t tile_chunk(int rho, int c, uint32_t half_byt
 // the lower original slot.
 __device__ __forceinline__ uint32_t key_low(int orig, int rho) { return ((0xFFFFu - (uint32_t)orig) << 16) | (uint32_t)rho; }
 
+// cos and -sin of 2*pi*(t/2^32) for two phases at once with packed fp32 arithmetic; the octant
+// reduction and the polynomials are those of sincos_phase, so each half gives the same bits.
+__device__ __forceinline__ void sincos_phase2(uint32_t ta, uint32_t tb, float2& cs, float2& nsn) {
+    const uint32_t ua = ta + 0x20000000u, ub = tb + 0x20000000u;
+    const float2 t = make_float2((float)((int)(ua & 0x3FFFFFFFu) - 0x20000000), (float)((int)(ub & 0x3FFFFFFFu) - 0x20000000));
+    const float2 y = __fmul2_rn(t, make_float2(1.862645149230957e-09f, 1.862645149230957e-09f));  // 2^-29
+    const float2 z = __fmul2_rn(y, y);
+    float2 p = __ffma2_rn(z, make_float2(-3.587714997811334e-05f, -3.587714997811334e-05f),
+                          make_float2(0.0024898717780787645f, 0.0024898717780787645f));
+    p = __ffma2_rn(z, p, make_float2(-0.08074536717605851f, -0.08074536717605851f));
+    p = __ffma2_rn(z, p, make_float2(0.7853981525308736f, 0.7853981525308736f));
+    const float2 sp = __fmul2_rn(y, p);
+    float2 c = __ffma2_rn(z, make_float2(-0.0003191315544232772f, -0.0003191315544232772f),
+                          make_float2(0.01585035496683941f, 0.01585035496683941f));
+    c = __ffma2_rn(z, c, make_float2(-0.308424473701413f, -0.308424473701413f));
+    c = __ffma2_rn(z, c, make_float2(1.0f, 1.0f));
+    // quarter turns: bit 30 of u swaps sine and cosine, bit 31 of u (of u + 2^30) flips the sine (cosine)
+    const bool swa = ua & 0x40000000u, swb = ub & 0x40000000u;
+    const uint32_t ca = __float_as_uint(swa ? sp.x : c.x), sa = __float_as_uint(swa ? c.x : sp.x);
+    const uint32_t cb = __float_as_uint(swb ? sp.y : c.y), sb = __float_as_uint(swb ? c.y : sp.y);
+    cs = make_float2(__uint_as_float(ca ^ ((ua + 0x40000000u) & 0x80000000u)),
+                     __uint_as_float(cb ^ ((ub + 0x40000000u) & 0x80000000u)));
+    nsn = make_float2(__uint_as_float(sa ^ (~ua & 0x80000000u)), __uint_as_float(sb ^ (~ub & 0x80000000u)));
+}
+
 // ---- the kernel ------------------------------------------------------------------------------------
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
@@ -219,13 +244,16 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         const int grp = lane >> 3, f0 = (lane & 7) * 8;
         const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
         const float inv = rsqrtf((float)kTcD);
-        float2 g[8];
+        // folded statistic g_f = c_f z(q)_f / sqrt(d), packed by frequency pairs (f, f+1)
+        float2 gx[4], gy[4], ngx[4];
         uint32_t phi_lo[8], phi_hi[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const float qr = q[f0 + u] * inv, qi = q[f0 + u + 64] * inv;
             const float2 c = tab.cw[f0 + u];
-            g[u] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+            const float x = c.x * qr - c.y * qi, y = c.x * qi + c.y * qr;
+            if (u & 1) { gx[u >> 1].y = x; gy[u >> 1].y = y; ngx[u >> 1].y = -x; }
+            else { gx[u >> 1].x = x; gy[u >> 1].x = y; ngx[u >> 1].x = -x; }
             phi_lo[u] = (uint32_t)tab.phi[f0 + u];
             phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
         }
@@ -252,26 +280,30 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
                 if (j < n) {
                     const uint4 wr = *reinterpret_cast<const uint4*>(tile + j * 256 + (lane & 7) * 16);
                     const uint4 wi = *reinterpret_cast<const uint4*>(tile + j * 256 + 128 + (lane & 7) * 16);
-                    const float kre[8] = {bf16lo(wr.x), bf16hi(wr.x), bf16lo(wr.y), bf16hi(wr.y),
-                                          bf16lo(wr.z), bf16hi(wr.z), bf16lo(wr.w), bf16hi(wr.w)};
-                    const float kim[8] = {bf16lo(wi.x), bf16hi(wi.x), bf16lo(wi.y), bf16hi(wi.y),
-                                          bf16lo(wi.z), bf16hi(wi.z), bf16lo(wi.w), bf16hi(wi.w)};
+                    const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
                     const long long dist = pref - (long long)spos[j];
                     const uint32_t dlo = (uint32_t)dist, dhi = (uint32_t)((unsigned long long)dist >> 32);
+                    float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const float tr = fmaf(g[u].x, kre[u], g[u].y * kim[u]);
-                        const float ti = fmaf(g[u].y, kre[u], -g[u].x * kim[u]);
+                    for (int p = 0; p < 4; ++p) {
+                        const float2 kre = make_float2(bf16lo(wre[p]), bf16hi(wre[p]));
+                        const float2 kim = make_float2(bf16lo(wim[p]), bf16hi(wim[p]));
+                        // t = g conj(k): real and imaginary part for the two frequencies of the pair
+                        const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
+                        const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
                         if (rotate) {
                             // bits 32..63 of dist * phi (mod 2^64)
-                            const uint32_t top = __umulhi(dlo, phi_lo[u]) + dlo * phi_hi[u] + dhi * phi_lo[u];
-                            float sn, cs;
-                            sincos_phase(top, sn, cs);
-                            acc += fmaf(tr, cs, -ti * sn);
+                            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + dhi * phi_lo[2 * p];
+                            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + dhi * phi_lo[2 * p + 1];
+                            float2 cs, nsn;
+                            sincos_phase2(ta, tb, cs, nsn);
+                            acc2 = __ffma2_rn(tr, cs, acc2);
+                            acc2 = __ffma2_rn(ti, nsn, acc2);
                         } else {
-                            acc += tr;
+                            acc2 = __fadd2_rn(acc2, tr);
                         }
                     }
+                    acc = acc2.x + acc2.y;
                 }
 #pragma unroll
                 for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);

@@ -183,6 +183,38 @@ akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t* lay, void
                                   int32_t* idx_sorted, int32_t* pick_order, float* pick_gain,
                                   float* scores, int32_t* n_kept, int32_t* status, void* stream);
 
+/*
+ * alpha_compress_event_static -- the same event as alpha_compress_event, for callers that must not
+ * allocate device memory. (The paper has no counterpart: this is a deployment variant, not a step
+ * of the method.)
+ *
+ * Who needs it: alpha_compress_event keeps the intermediate scores of an event that does not fit
+ * on chip in the handle's scratch, which it grows with cudaMalloc (plus a device-wide synchronise
+ * when it regrows). A serving process whose memory pool has already reserved the whole device
+ * cannot afford that call failing, and a latency-critical decode thread cannot afford its implicit
+ * synchronisation. This entry point calls no cudaMalloc, cudaFree or other allocating routine: the
+ * scores go to an array of AKV_STATIC_SCORES_MAX floats (4 MiB) that is part of the library image,
+ * so every GPU that loads the library holds those 4 MiB until the process exits.
+ *
+ *   - It always runs as three launches (score, select, compact) on `stream`; results are those
+ *     of alpha_compress_event on the same route.
+ *   - Limit: B*L*H*N <= AKV_STATIC_SCORES_MAX, otherwise AKV_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current). Make that first call before starting any stream capture.
+ *   - All calls on one device share the array and it keeps the previous call's scores. Nothing in
+ *     it has to start at zero (each call writes every score it later reads), but two calls whose
+ *     kernels overlap on the GPU (different streams, no ordering between them) race on it: order
+ *     such calls yourself.
+ * Arguments as alpha_compress_event, without the `scores` output.
+ */
+#define AKV_STATIC_SCORES_MAX (1u << 20)
+akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                         int64_t pos_stride_b, int64_t pos_stride_l, int64_t pos_stride_h,
+                                         const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
+                                         const float* flat_sig, int32_t budget, const akv_options_t* opt,
+                                         int32_t* idx_sorted, int32_t* pick_order, float* pick_gain,
+                                         int32_t* n_kept, int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

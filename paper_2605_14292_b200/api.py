@@ -25,7 +25,7 @@ FLAG_NO_PRUNE = 2
 
 EXPORTS = ("akv_default_options", "akv_create", "akv_destroy", "akv_last_error", "akv_status_string",
            "akv_launch_count", "alpha_score", "alpha_select", "alpha_signature_flat", "kv_compact",
-           "alpha_compress_event")
+           "alpha_compress_event", "alpha_compress_event_static")
 
 
 class AkvError(RuntimeError):
@@ -72,6 +72,8 @@ def load_library(path: Optional[str] = None):
     lib.kv_compact.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, i32, vp]
     lib.alpha_compress_event.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32,
                                          C.POINTER(_Options), vp, vp, vp, vp, vp, vp, vp]
+    lib.alpha_compress_event_static.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32,
+                                                C.POINTER(_Options), vp, vp, vp, vp, vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -309,6 +311,31 @@ def alpha_compress_event(K, V, pos, qstat, budget: int, opts: Optional[Options] 
             _handle(K.device), C.byref(lay.c()), _ptr(K), _ptr(V), _ptr(pos), sb, sl, sh, _ptr(n_cand), _ptr(qstat),
             _ptr(p_ref), _ptr(flat_sig), budget, C.byref(opts.c()), _ptr(sel.idx_sorted), _ptr(sel.pick_order),
             _ptr(sel.pick_gain), _ptr(sel.scores), _ptr(sel.n_kept), _ptr(sel.status), _stream()))
+    return sel
+
+
+STATIC_SCORES_MAX = 1 << 20
+
+
+def alpha_compress_event_static(K, V, pos, qstat, budget: int, opts: Optional[Options] = None, p_ref=None, n_cand=None,
+                                flat_sig=None, layout: Optional[Layout] = None, detail: bool = True,
+                                out: Optional[Selection] = None) -> Selection:
+    """The compression event for callers that must not allocate device memory -- C entry point
+    ``alpha_compress_event_static``. Scores are kept in a 4 MiB array inside the library image instead of
+    cudaMalloc'ed scratch, so B*L*H*N may not exceed STATIC_SCORES_MAX; calls on one device share that array
+    and must not overlap on the GPU. Pass ``out`` (pre-allocated outputs) to keep torch from allocating too.
+    K, V and pos are rewritten in place."""
+    lay = _lay(K, layout)
+    opts = opts or Options()
+    _need(qstat, torch.float32, "qstat"); _need(p_ref, torch.int32, "p_ref"); _need(n_cand, torch.int32, "n_cand")
+    _need(flat_sig, torch.float32, "flat_sig")
+    sel = out or _alloc_sel(lay, budget, K.device, detail)
+    sb, sl, sh = _pos_strides(pos, lay)
+    with torch.cuda.device(K.device):
+        _check(load_library().alpha_compress_event_static(
+            _handle(K.device), C.byref(lay.c()), _ptr(K), _ptr(V), _ptr(pos), sb, sl, sh, _ptr(n_cand), _ptr(qstat),
+            _ptr(p_ref), _ptr(flat_sig), budget, C.byref(opts.c()), _ptr(sel.idx_sorted), _ptr(sel.pick_order),
+            _ptr(sel.pick_gain), _ptr(sel.n_kept), _ptr(sel.status), _stream()))
     return sel
 
 

@@ -483,3 +483,73 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     c.lay = a.lay; c.K = K; c.V = V; c.pos = a.pos; c.idx_sorted = idx_sorted; c.budget = budget;
     return launch_compact(h, c, st);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Three-launch event with the intermediate scores in library-owned static device memory.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+static __device__ __align__(256) float g_static_scores[AKV_STATIC_SCORES_MAX];
+
+// In host code `g_static_scores` is only a stand-in for the symbol; the device address comes from
+// the runtime, once per device, with that device current.
+static akv_status_t static_scores_address(int device, float** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static float* addr[kMaxDevices] = {};
+    if (device < 0 || device >= kMaxDevices) return fail(AKV_ERR_UNSUPPORTED, "device %d: at most %d devices", device, kMaxDevices);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[device]) {
+        void* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scores));
+        addr[device] = static_cast<float*>(p);
+    }
+    *out = addr[device];
+    return AKV_OK;
+}
+
+extern "C" akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V,
+                                                    int32_t* pos, int64_t psb, int64_t psl, int64_t psh,
+                                                    const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
+                                                    const float* flat_sig, int32_t budget, const akv_options_t* opt,
+                                                    int32_t* idx_sorted, int32_t* pick_order, float* pick_gain,
+                                                    int32_t* n_kept, int32_t* status, void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_compress_event_static: handle is NULL");
+    EventArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if ((s = check_budget(budget, lay->N)) != AKV_OK) return s;
+    if (!K || !V || !qstat || !idx_sorted)
+        return fail(AKV_ERR_INVALID_ARG, "alpha_compress_event_static: K, V, qstat and idx_sorted must not be NULL");
+    if (!aligned16(K) || !aligned16(V)) return fail(AKV_ERR_ALIGNMENT, "alpha_compress_event_static: K/V must be 16-byte aligned");
+    const unsigned long long need = (unsigned long long)lay->B * lay->L * lay->H * lay->N;
+    if (need > AKV_STATIC_SCORES_MAX)
+        return fail(AKV_ERR_WORKSPACE, "alpha_compress_event_static: B*L*H*N = %llu scores exceed the static scratch of %llu",
+                    need, (unsigned long long)AKV_STATIC_SCORES_MAX);
+    if ((s = check_pos_written(a.lay, pos, psb, psl, psh)) != AKV_OK) return s;
+    if ((s = fill_select_args(a, opt, V, flat_sig)) != AKV_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    float* scratch = nullptr;
+    if ((s = static_scores_address(h->device, &scratch)) != AKV_OK) return s;
+    build_tables(h, lay->d, opt->rope_base, opt->future_window);
+    cudaStream_t st = (cudaStream_t)stream;
+    a.K = K; a.V = V;
+    a.pos = PosDesc{pos, psb, psl, psh};
+    a.n_cand = n_cand; a.qstat = qstat; a.p_ref = p_ref;
+    a.budget = budget;
+    a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
+    a.scores = scratch; a.n_kept = n_kept; a.status = status;
+    // Every score the selection reads (slots below n_cand) is written by the scoring launch of this
+    // same call, so nothing left in the array by an earlier call needs clearing.
+    EventArgs sa = a;
+    sa.status = nullptr;  // the selection kernel writes the final status word
+    if ((s = launch_score(h, sa, st)) != AKV_OK) return s;
+    if ((s = launch_select(h, a, st)) != AKV_OK) return s;
+    CompactArgs c;
+    memset(&c, 0, sizeof(c));
+    c.lay = a.lay; c.K = K; c.V = V; c.pos = a.pos; c.idx_sorted = idx_sorted; c.budget = budget;
+    return launch_compact(h, c, st);
+}

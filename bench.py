@@ -37,7 +37,7 @@ def algorithmic_bytes(N, b, d, esize):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on this workload, from
 # the ncu capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 311380224 + 99654400
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def load_peaks():
@@ -243,7 +243,7 @@ def run_gpu(args):
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
-                "kernel": "event_tc_kernel<fused>", "algorithmic_bytes_per_launch": bytes_per_launch}
+                "kernel": "event_tri_kernel<fused>", "algorithmic_bytes_per_launch": bytes_per_launch}
 
     # end to end: pinned host buffers -> device, the same C-ABI call, indices and kept counts back
     hK, hV, hP = (torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (K0, V0, P0))

@@ -1,0 +1,526 @@
+// Fast event kernel for bf16, d = 128, per-head signatures, N <= 256, used when the pool that
+// survives pruning is expected to stay within 128 rows (N <= 128 or budget <= 64). One CTA of four
+// warps per event, four CTAs resident per SM.
+//
+//   1. K rows arrive in shared memory by per-row bulk copies (cp.async.bulk + mbarrier) and are
+//      scored there (fused RoPE rotate-and-dot against the folded query statistic).
+//   2. Only candidates with  s_i >= s_(b) - lambda * (1 + slack)  can ever be an argmax of Eq. 2
+//      (the running maximum m never exceeds 1, so every still unchosen member of the top-b scores
+//      beats the others). s_(b) comes from a bisection over the score keys; that pool of P rows,
+//      in slot order, is the only part of V that is read for the selection.
+//   3. P <= 128: the pool's V rows form a K-major, 128-byte-swizzled operand tile, one
+//      tcgen05.mma sequence writes the pool's cosine matrix (raw dot products, fp32) into tensor
+//      memory, and the four warps move its lower triangle to shared memory (tcgen05.ld), taking
+//      the squared norms of Eq. 1 from the diagonal on the way.
+//      P > 128 (hardly any pruning): no tensor-core product; rows of the cosine matrix are plain
+//      dot products from the V tile, one picked row at a time.
+//   4. Algorithm 1 runs in ONE warp: every lane owns up to P/32 candidates and keeps s, the
+//      running maximum and lambda/norm in registers; the argmax is two warp reductions, the picked
+//      row of the cosine matrix is read from the triangle without bank conflicts.
+//   5. Kept rows are written back in place: K, V and positions are re-read (L2) and held on chip
+//      before the first store.
+#pragma once
+#include "akv_event_tc.cuh"
+
+namespace akv {
+
+struct TriSmem {
+    unsigned tile, s, key, spos, bypool, taken, order, gain, idx, row, misc, total;
+    int tile_rows;
+};
+// Layout after the 1024-byte aligned base. `key` (score keys) and `r` (reciprocal norms) share storage.
+__host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
+    TriSmem p;
+    p.tile_rows = ((N + 15) & ~15) < 128 ? 128 : ((N + 15) & ~15);
+    const unsigned np = (unsigned)((N + 3) & ~3);
+    unsigned o = 0;
+    p.tile = o;   o += (unsigned)p.tile_rows * 256u < 33792u ? 33792u : (unsigned)p.tile_rows * 256u;  // >= triangle of 128 rows
+    p.s = o;      o += align16(np * 4);
+    p.key = o;    o += align16(np * 4);
+    p.spos = o;   o += align16(np * 4);
+    p.bypool = o; o += align16(np * 2);
+    p.taken = o;  o += align16(np);
+    p.order = o;  o += align16((unsigned)budget * 4);
+    p.gain = o;   o += align16((unsigned)budget * 4);
+    p.idx = o;    o += align16((unsigned)budget * 4);
+    p.row = o;    o += 2 * 1024;  // two rows of the cosine matrix (plain-dot route), 256 floats each
+    p.misc = o;   o += 64;        // mbarriers (2 x 8), tmem base, pool size, block-max scratch
+    p.total = o + 1024;           // room to align the base to 1024 bytes
+    return p;
+}
+
+// 32 consecutive columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// entry (a, b), a >= b, of a lower triangle stored row by row; rows a = lane + 32 k of one warp
+// fall into 32 different banks for a fixed b, and so do consecutive b for a fixed a
+__device__ __forceinline__ int tri_row(int a) { return (a * (a + 1)) >> 1; }
+
+// Score terms of one key row for the 8 frequencies a lane covers, packed by frequency pairs.
+// wr / wi: real and imaginary halves (8 bf16 each); returns the lane's partial sum.
+template <bool ROTATE>
+__device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, const float2 (&gx)[4], const float2 (&gy)[4],
+                                             const float2 (&ngx)[4], const uint32_t (&phi_lo)[8], const uint32_t (&phi_hi)[8],
+                                             uint32_t dlo, uint32_t dhi) {
+    const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
+    float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        const float2 kre = make_float2(bf16lo(wre[p]), bf16hi(wre[p]));
+        const float2 kim = make_float2(bf16lo(wim[p]), bf16hi(wim[p]));
+        // t = g conj(k): real and imaginary part for the two frequencies of the pair
+        const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
+        if (ROTATE) {
+            const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
+            // bits 32..63 of dist * phi (mod 2^64); dhi is 0 or all ones
+            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + (dhi & (0u - phi_lo[2 * p]));
+            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + (dhi & (0u - phi_lo[2 * p + 1]));
+            float2 cs, nsn;
+            sincos_phase2(ta, tb, cs, nsn);
+            acc2 = __ffma2_rn(tr, cs, acc2);
+            acc2 = __ffma2_rn(ti, nsn, acc2);
+        } else {
+            acc2 = __fadd2_rn(acc2, tr);
+        }
+    }
+    return acc2.x + acc2.y;
+}
+
+// Per-lane state of the single-warp greedy loop: candidates rho = lane + 32 k, k < CPL.
+template <int CPL>
+struct GreedyLane {
+    float sv[CPL], lr[CPL], M[CPL];
+    uint32_t alive;
+    __device__ __forceinline__ void init(int lane, int P, const float* s, const unsigned short* bypool, const float* r, float lam,
+                                         bool use_r) {
+        alive = 0u;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            const int rho = lane + 32 * k;
+            sv[k] = 0.f; lr[k] = 0.f; M[k] = 0.f;
+            if (rho < P) {
+                sv[k] = s[bypool[rho]];
+                lr[k] = use_r ? lam * r[rho] : 0.f;
+                alive |= 1u << k;
+            }
+        }
+    }
+    // a = s - lambda m over the candidates still alive; returns the key of the best one and its pool
+    // row (ties to the lower row, which is the lower slot); the owner drops it from its alive set
+    __device__ __forceinline__ int pick(int lane, uint32_t& best_key) {
+        uint32_t bk = 0u;
+        int brho = 0;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            const uint32_t key = ((alive >> k) & 1u) ? orderable(fmaf(-lr[k], M[k], sv[k])) : 0u;
+            if (key > bk) { bk = key; brho = lane + 32 * k; }
+        }
+        const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, bk);
+        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, (bk == whi && bk != 0u) ? 0xFFFFu - (uint32_t)brho : 0u);
+        const int irho = (int)(0xFFFFu - wlo);
+        if ((irho & 31) == lane) alive &= ~(1u << (irho >> 5));
+        best_key = whi;
+        return irho;
+    }
+};
+
+// The loop of Algorithm 1 run by one warp without any block-wide barrier. with_sims: the running
+// maximum is updated from the triangle `tri` of raw dot products (needs P <= 128 and r); otherwise
+// the picks are the plain arg-max sequence (top-k in pick order).
+template <int CPL>
+__device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bool with_sims, const float* s,
+                                                  const unsigned short* bypool, const float* r, float lam, const float* tri,
+                                                  uint32_t* park_key, int* park_row) {
+    GreedyLane<CPL> g;
+    g.init(lane, P, s, bypool, r, lam, with_sims);
+    int trow[CPL];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) trow[k] = tri_row(lane + 32 * k);
+    for (int t = 0; t < picks; ++t) {
+        uint32_t bk;
+        const int irho = g.pick(lane, bk);
+        if (lane == 0) { park_key[t] = bk; park_row[t] = irho; }
+        if (!with_sims || t + 1 == picks) continue;
+        // m <- max(m, Sims[i, :]) from the triangle: entry (max, min)
+        const float ri = r[irho];
+        const int ti = tri_row(irho);
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            const int rho = lane + 32 * k;
+            if (rho < P) g.M[k] = fmaxf(g.M[k], ri * tri[rho > irho ? trow[k] + irho : ti + rho]);
+        }
+    }
+}
+
+// FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
+// nothing is rewritten).
+template <bool FUSED>
+__global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int n = event_n(a, id.b);
+    const int N = lay.N;
+    const int picks = min(a.budget, n);
+    const TriSmem sp = plan_tri_smem(N, a.budget);
+    unsigned char* tile = smem + sp.tile;
+    float* tri = reinterpret_cast<float*>(tile);  // lower triangle of the cosine matrix, after the product
+    float* s = reinterpret_cast<float*>(smem + sp.s);
+    uint32_t* key = reinterpret_cast<uint32_t*>(smem + sp.key);
+    float* r = reinterpret_cast<float*>(smem + sp.key);  // reuses the score keys' storage
+    int* spos = reinterpret_cast<int*>(smem + sp.spos);
+    unsigned short* bypool = reinterpret_cast<unsigned short*>(smem + sp.bypool);
+    unsigned char* taken = smem + sp.taken;
+    int* order = reinterpret_cast<int*>(smem + sp.order);
+    float* gain = reinterpret_cast<float*>(smem + sp.gain);
+    int* idx = reinterpret_cast<int*>(smem + sp.idx);
+    float* rowbuf = reinterpret_cast<float*>(smem + sp.row);
+    const uint32_t barK = smem_u32(smem + sp.misc);
+    const uint32_t barM = barK + 8;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 16);
+    int* pool_holder = reinterpret_cast<int*>(smem + sp.misc + 20);
+    int* pick_holder = reinterpret_cast<int*>(smem + sp.misc + 24);
+    int* redi = reinterpret_cast<int*>(smem + sp.misc + 32);
+    const uint32_t tile_u32 = smem_u32(tile);
+    const uint32_t half_bytes = (uint32_t)sp.tile_rows * 128u;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool similarity = a.greedy != 0;
+    const int np4 = (N + 3) & ~3;
+    // row addressing: dense events are one base offset plus a row stride
+    const bool dense = lay.page_size == 0;
+    const long long ev_off = dense ? id.b * lay.sb + id.l * lay.sl + id.h * lay.sh : 0;
+    auto rowoff = [&](int j) -> long long {
+        return dense ? ev_off + (long long)j * lay.sn : row_offset(lay, id.b, id.l, id.h, j);
+    };
+    __nv_bfloat16* Kg = reinterpret_cast<__nv_bfloat16*>(a.K);
+    __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
+
+    // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
+    // next CTA of this kernel only after that, so a late allocation would serialise the CTAs.
+    const bool use_tc = similarity;
+    if (tid == 0) {
+        mbar_init(barK, 1);
+        mbar_init(barM, 1);
+        mbar_init_fence();
+    }
+    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), kTcCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = use_tc ? *tmem_holder : 0u;
+
+    // ---- scores ---------------------------------------------------------------------------------
+    int bad = 0;
+    int timeout = 0;
+    if (FUSED) {
+        if (tid == 0) mbar_expect_tx(barK, (uint32_t)n * 256u);
+        for (int row = tid; row < n; row += kTcThreads) bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), 256u, barK);
+        const int* gpos = event_pos(a.pos, id);
+        const bool rotate = gpos != nullptr;
+        int pmax = INT_MIN;
+        for (int j = tid; j < n; j += kTcThreads) {
+            const int p = rotate ? gpos[j] : 0;
+            spos[j] = p;
+            pmax = max(pmax, p);
+        }
+        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
+        const int grp = lane >> 3, f0 = (lane & 7) * 8;
+        const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
+        const float inv = rsqrtf((float)kTcD);
+        // folded statistic g_f = c_f z(q)_f / sqrt(d), packed by frequency pairs (f, f+1)
+        float2 gx[4], gy[4], ngx[4];
+        uint32_t phi_lo[8], phi_hi[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float qr = q[f0 + u] * inv, qi = q[f0 + u + 64] * inv;
+            const float2 c = tab.cw[f0 + u];
+            const float x = c.x * qr - c.y * qi, y = c.x * qi + c.y * qr;
+            if (u & 1) { gx[u >> 1].y = x; gy[u >> 1].y = y; ngx[u >> 1].y = -x; }
+            else { gx[u >> 1].x = x; gy[u >> 1].x = y; ngx[u >> 1].x = -x; }
+            phi_lo[u] = (uint32_t)tab.phi[f0 + u];
+            phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
+        }
+        long long pref = 0;
+        if (rotate && !a.p_ref) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
+            if (lane == 0) redi[warp] = pmax;
+        }
+        __syncthreads();
+        if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
+        timeout = !mbar_wait_bounded(barK, 0);
+        if (!timeout) {
+            for (int j0 = 4 * warp; j0 < n; j0 += 4 * (kTcThreads / 32)) {
+                const int j = j0 + grp;
+                float acc = 0.f;
+                if (j < n) {
+                    const uint4 wr = *reinterpret_cast<const uint4*>(tile + j * 256 + (lane & 7) * 16);
+                    const uint4 wi = *reinterpret_cast<const uint4*>(tile + j * 256 + 128 + (lane & 7) * 16);
+                    if (rotate) {
+                        const long long dist = pref - (long long)spos[j];
+                        acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
+                                                (uint32_t)((unsigned long long)dist >> 32));
+                    } else {
+                        acc = score_lane8<false>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, 0u, 0u);
+                    }
+                }
+#pragma unroll
+                for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+                if (j < n && (lane & 7) == 0) {
+                    if (a.scores) a.scores[(long long)id.e * N + j] = acc;
+                    const bool fin = isfinite(acc);
+                    bad |= !fin;
+                    const float sj = fin ? acc : -INFINITY;
+                    s[j] = sj;
+                    key[j] = orderable(sj);
+                }
+            }
+        }
+    } else {
+        for (int j = tid; j < n; j += kTcThreads) {
+            const float sc = a.scores[(long long)id.e * N + j];
+            const bool fin = isfinite(sc);
+            bad |= !fin;
+            const float sj = fin ? sc : -INFINITY;
+            s[j] = sj;
+            key[j] = orderable(sj);
+        }
+    }
+    for (int j = n + tid; j < np4; j += kTcThreads) key[j] = 0u;  // below every real key
+    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
+    timeout = __syncthreads_or(timeout);
+    if (timeout) {
+        if (tid == 0 && a.status) a.status[id.e] = 3;
+        mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
+        if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
+        return;
+    }
+    bad = __syncthreads_or(bad);
+
+    // ---- s_(b) by bisection over the score keys, then the pool in slot order (warp 0) -------------
+    if (warp == 0) {
+        uint32_t kk[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int j = lane + 32 * k;
+            kk[k] = j < np4 ? key[j] : 0u;
+        }
+        uint32_t kb = 0u;  // the picks-th largest key: the largest v with at least `picks` keys >= v
+        if (picks > 0) {
+            for (int bit = 31; bit >= 0; --bit) {
+                const uint32_t v = kb | (1u << bit);
+                int cnt = 0;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) cnt += kk[k] >= v;
+                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= picks) kb = v;
+            }
+        }
+        const float sb = from_orderable(kb);
+        // -inf keeps everyone
+        const float thr = a.no_prune ? -INFINITY : fmaf(-1.001f, a.lam, sb) - 1e-6f * fabsf(sb);
+        int base = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const bool in = kk[k] != 0u && (similarity ? !(from_orderable(kk[k]) < thr) : kk[k] >= kb);
+            const uint32_t mask = __ballot_sync(0xFFFFFFFFu, in);
+            if (in) bypool[base + __popc(mask & ((1u << lane) - 1u))] = (unsigned short)(lane + 32 * k);
+            base += __popc(mask);
+        }
+        if (lane == 0) *pool_holder = base;
+    }
+    __syncthreads();  // every key has been read: its storage becomes r below
+    const int P = *pool_holder;
+    const bool fast = similarity && P <= 128 && picks > 1;
+    const bool slow = similarity && P > 128;
+
+    // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
+    if (similarity) {
+        for (int x = tid; x < P * 16; x += kTcThreads) {
+            const int rho = x >> 4, c = x & 15;
+            cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(bypool[rho]) + c * 8);
+        }
+        cp_async_wait_all();
+        fence_proxy_async();
+        __syncthreads();
+    }
+    if (fast) {
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t idesc = umma_idesc_bf16(128, (P + 15) & ~15);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
+                umma_bf16(tbase, umma_desc_sw128(tile_u32 + koff), umma_desc_sw128(tile_u32 + koff), idesc, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(barM);
+        }
+        timeout = !mbar_wait_bounded(barM, 0);
+        tc_fence_after();
+    }
+    timeout = __syncthreads_or(timeout);  // also: the product has read the whole tile before the triangle lands on it
+    if (timeout) {
+        if (tid == 0 && a.status) a.status[id.e] = 3;
+        if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
+        return;
+    }
+    if (fast) {
+        // lower triangle -> shared memory; row rho = 32 warp + lane needs columns 0..rho
+        const int rho = 32 * warp + lane;
+        if (32 * warp < P) {
+            float diag = 1.f;
+            const int trow = tri_row(rho);
+            for (int cb = 0; cb <= warp; ++cb) {
+                uint32_t v[32];
+                tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * cb), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    const int c = 32 * cb + k;
+                    if (c <= rho && rho < P) tri[trow + c] = __uint_as_float(v[k]);
+                    if (c == rho) diag = __uint_as_float(v[k]);
+                }
+            }
+            if (rho < P) r[rho] = 1.f / (sqrtf(diag) + a.eps);
+        }
+    } else if (slow) {
+        // reciprocal norms from the tile (Eq. 1)
+        for (int rho = tid; rho < P; rho += kTcThreads) {
+            float ss = 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                float x[8];
+                load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho, c, half_bytes)), x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
+            }
+            r[rho] = 1.f / (sqrtf(ss) + a.eps);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
+
+    // ---- Algorithm 1 in warp 0 -------------------------------------------------------------------------
+    // The winning key of every pick is parked in gain[] and its pool row in order[]; both are decoded
+    // after the loop.
+    uint32_t* park_key = reinterpret_cast<uint32_t*>(gain);
+    if (!slow) {
+        if (warp == 0) {
+            if (P <= 128) picks_in_one_warp<4>(lane, P, picks, fast, s, bypool, r, a.lam, tri, park_key, order);
+            else picks_in_one_warp<8>(lane, P, picks, false, s, bypool, r, a.lam, tri, park_key, order);
+        }
+    } else {
+        GreedyLane<8> g;
+        if (warp == 0) g.init(lane, P, s, bypool, r, a.lam, true);
+        for (int t = 0; t < picks; ++t) {
+            if (warp == 0) {
+                uint32_t bk;
+                const int irho = g.pick(lane, bk);
+                if (lane == 0) { park_key[t] = bk; order[t] = irho; *pick_holder = irho; }
+            }
+            if (t + 1 == picks) break;
+            __syncthreads();
+            const int irho = *pick_holder;
+            // row irho of the cosine matrix by plain dot products from the tile
+            for (int rho = tid; rho < P; rho += kTcThreads) {
+                float acc = 0.f;
+#pragma unroll 4
+                for (int c = 0; c < 16; ++c) {
+                    float vi[8], vj[8];
+                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(irho, c, half_bytes)), vi);
+                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho, c, half_bytes)), vj);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc = fmaf(vi[e], vj[e], acc);
+                }
+                rowbuf[rho] = acc;
+            }
+            __syncthreads();
+            if (warp == 0) {
+                const float ri = r[irho];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int rho = lane + 32 * k;
+                    if (rho < P) g.M[k] = fmaxf(g.M[k], ri * rowbuf[rho]);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int t = tid; t < picks; t += kTcThreads) {
+        const int j = bypool[order[t]];
+        gain[t] = from_orderable(park_key[t]);
+        order[t] = j;
+        taken[j] = 1;
+    }
+    __syncthreads();
+
+    // ---- sort(S) and outputs -------------------------------------------------------------------------
+    ordered_indices(n, a.budget, taken, idx);
+    __syncthreads();
+    const long long ob = (long long)id.e * a.budget;
+    for (int t = tid; t < a.budget; t += kTcThreads) {
+        a.idx_sorted[ob + t] = idx[t];
+        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
+        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
+    }
+    if (tid == 0) {
+        if (a.n_kept) a.n_kept[id.e] = picks;
+        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+    }
+    if (!FUSED) return;
+
+    // ---- compaction in place ----------------------------------------------------------------------
+    // Every kept K and V row and position is on chip (registers for up to 64 rows, else the tile)
+    // before the first store: a destination slot can be another kept row's source.
+    int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
+    if (picks <= 64) {
+        uint4 kreg[8], vreg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int x = tid + i * kTcThreads;
+            if (x < picks * 16) {
+                const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
+                kreg[i] = *reinterpret_cast<const uint4*>(Kg + off);
+                vreg[i] = *reinterpret_cast<const uint4*>(Vg + off);
+            }
+        }
+        __syncthreads();  // every load above has been performed
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int x = tid + i * kTcThreads;
+            if (x < picks * 16) {
+                const long long off = rowoff(x >> 4) + (x & 15) * 8;
+                *reinterpret_cast<uint4*>(Kg + off) = kreg[i];
+                *reinterpret_cast<uint4*>(Vg + off) = vreg[i];
+            }
+        }
+    } else {
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            __nv_bfloat16* X = pass ? Vg : Kg;
+            __syncthreads();  // the tile is free (greedy loop, or the previous pass, is done with it)
+            for (int x = tid; x < picks * 16; x += kTcThreads)
+                copy16(tile + x * 16, reinterpret_cast<const char*>(X + rowoff(idx[x >> 4])) + (x & 15) * 16);
+            __syncthreads();
+            for (int x = tid; x < picks * 16; x += kTcThreads)
+                copy16(reinterpret_cast<char*>(X + rowoff(x >> 4)) + (x & 15) * 16, tile + x * 16);
+        }
+    }
+    if (wpos)
+        for (int t = tid; t < picks; t += kTcThreads) wpos[t] = spos[idx[t]];
+}
+
+}  // namespace akv

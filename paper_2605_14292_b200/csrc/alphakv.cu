@@ -8,7 +8,7 @@
 #include <cstdio>
 #include <cstring>
 
-#include "akv_event_tc.cuh"
+#include "akv_event_tri.cuh"
 
 using namespace akv;
 
@@ -287,7 +287,24 @@ static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t s
     return launched(FUSED ? "event_tc" : "select_tc");
 }
 
+// Single-warp greedy loop over a triangle of the pool's cosine matrix: the shapes whose pruned pool
+// normally stays within 128 rows.
+static bool tri_path_ok(const EventArgs& a) { return tc_path_ok(a) && (a.lay.N <= 128 || a.budget <= 64); }
+template <bool FUSED>
+static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    const TriSmem sp = plan_tri_smem(a.lay.N, a.budget);
+    if ((int)sp.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "budget %d needs too much shared memory", a.budget);
+    akv_status_t s;
+    if ((s = set_smem(event_tri_kernel<FUSED>, sp.total)) != AKV_OK) return s;
+    CUDA_TRY(cudaFuncSetAttribute(event_tri_kernel<FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                  (int)cudaSharedmemCarveoutMaxShared));
+    event_tri_kernel<FUSED><<<E, kTcThreads, sp.total, st>>>(a, h->tab);
+    return launched(FUSED ? "event_tri" : "select_tri");
+}
+
 static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    if (tri_path_ok(a) && a.V) return launch_tri<false>(h, a, st);
     if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st);
     return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st) : launch_select_t<float>(h, a, st);
 }
@@ -452,6 +469,7 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
     a.scores = scores; a.n_kept = n_kept; a.status = status;
 
+    if (tri_path_ok(a)) return launch_tri<true>(h, a, st);
     if (tc_path_ok(a)) return launch_tc<true>(h, a, st);
     const int es = lay->dtype == AKV_BF16 ? 2 : 4;
     const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);

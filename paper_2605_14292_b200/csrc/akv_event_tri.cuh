@@ -226,8 +226,20 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     int bad = 0;
     int timeout = 0;
     if (FUSED) {
-        if (tid == 0) mbar_expect_tx(barK, (uint32_t)n * 256u);
-        for (int row = tid; row < n; row += kTcThreads) bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), 256u, barK);
+        // K rows -> tile: one bulk copy when the event's rows are contiguous, one per page when pages
+        // are, else one per row; all issued by one thread (a bulk copy is a per-warp instruction)
+        if (tid == 0) {
+            mbar_expect_tx(barK, (uint32_t)n * 256u);
+            if (dense && lay.sn == kTcD) {
+                for (int row = 0; row < n; row += 128)  // 32 KB pieces
+                    bulk_g2s(tile_u32 + row * 256, Kg + ev_off + (long long)row * kTcD, (uint32_t)min(128, n - row) * 256u, barK);
+            } else if (!dense && lay.s_page_n == kTcD) {
+                for (int row = 0; row < n; row += lay.page_size)
+                    bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), (uint32_t)min(lay.page_size, n - row) * 256u, barK);
+            } else {
+                for (int row = 0; row < n; ++row) bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), 256u, barK);
+            }
+        }
         const int* gpos = event_pos(a.pos, id);
         const bool rotate = gpos != nullptr;
         int pmax = INT_MIN;

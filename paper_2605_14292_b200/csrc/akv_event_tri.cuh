@@ -101,35 +101,40 @@ __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, c
 template <int CPL>
 struct GreedyLane {
     float sv[CPL], lr[CPL], M[CPL];
-    uint32_t alive;
+    uint32_t am[CPL];  // all ones while the candidate competes; 0 once chosen, or when the row is empty
     __device__ __forceinline__ void init(int lane, int P, const float* s, const unsigned short* bypool, const float* r, float lam,
                                          bool use_r) {
-        alive = 0u;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
             const int rho = lane + 32 * k;
-            sv[k] = 0.f; lr[k] = 0.f; M[k] = 0.f;
+            sv[k] = 0.f; lr[k] = 0.f; M[k] = 0.f; am[k] = 0u;
             if (rho < P) {
                 sv[k] = s[bypool[rho]];
                 lr[k] = use_r ? lam * r[rho] : 0.f;
-                alive |= 1u << k;
+                am[k] = 0xFFFFFFFFu;
             }
         }
     }
-    // a = s - lambda m over the candidates still alive; returns the key of the best one and its pool
-    // row (ties to the lower row, which is the lower slot); the owner drops it from its alive set
+    // a = s - lambda m over the candidates still competing; returns the key of the best one and its
+    // pool row (ties to the lower row, which is the lower slot) and retires it
     __device__ __forceinline__ int pick(int lane, uint32_t& best_key) {
-        uint32_t bk = 0u;
-        int brho = 0;
+        uint32_t key[CPL];
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
-            const uint32_t key = ((alive >> k) & 1u) ? orderable(fmaf(-lr[k], M[k], sv[k])) : 0u;
-            if (key > bk) { bk = key; brho = lane + 32 * k; }
+            const uint32_t u = __float_as_uint(fmaf(-lr[k], M[k], sv[k]));
+            key[k] = (u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u)) & am[k];  // orderable(a), 0 when retired
         }
+        uint32_t bk = key[0];
+#pragma unroll
+        for (int k = 1; k < CPL; ++k) bk = max(bk, key[k]);
+        int kk = CPL - 1;
+#pragma unroll
+        for (int k = CPL - 2; k >= 0; --k) kk = key[k] == bk ? k : kk;
         const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, bk);
-        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, (bk == whi && bk != 0u) ? 0xFFFFu - (uint32_t)brho : 0u);
+        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, bk == whi ? 0xFFFFu - (uint32_t)(lane + 32 * kk) : 0u);
         const int irho = (int)(0xFFFFu - wlo);
-        if ((irho & 31) == lane) alive &= ~(1u << (irho >> 5));
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) am[k] = (lane + 32 * k == irho) ? 0u : am[k];
         best_key = whi;
         return irho;
     }
@@ -144,9 +149,10 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
                                                   uint32_t* park_key, int* park_row) {
     GreedyLane<CPL> g;
     g.init(lane, P, s, bypool, r, lam, with_sims);
-    int trow[CPL];
+    const char* tb = reinterpret_cast<const char*>(tri);
+    int trowB[CPL];  // byte offset of row rho of the triangle
 #pragma unroll
-    for (int k = 0; k < CPL; ++k) trow[k] = tri_row(lane + 32 * k);
+    for (int k = 0; k < CPL; ++k) trowB[k] = 4 * tri_row(lane + 32 * k);
     for (int t = 0; t < picks; ++t) {
         uint32_t bk;
         const int irho = g.pick(lane, bk);
@@ -154,11 +160,14 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
         if (!with_sims || t + 1 == picks) continue;
         // m <- max(m, Sims[i, :]) from the triangle: entry (max, min)
         const float ri = r[irho];
-        const int ti = tri_row(irho);
+        const int tiB = 4 * tri_row(irho), irho4 = 4 * irho;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
             const int rho = lane + 32 * k;
-            if (rho < P) g.M[k] = fmaxf(g.M[k], ri * tri[rho > irho ? trow[k] + irho : ti + rho]);
+            if (rho < P) {
+                const int off = rho > irho ? trowB[k] + irho4 : tiB + 4 * rho;
+                g.M[k] = fmaxf(g.M[k], ri * *reinterpret_cast<const float*>(tb + off));
+            }
         }
     }
 }

@@ -25,7 +25,7 @@
 namespace akv {
 
 struct TriSmem {
-    unsigned tile, s, key, spos, bypool, taken, order, gain, idx, row, misc, total;
+    unsigned tile, s, key, spos, bypool, taken, order, gain, idx, row, sect, misc, total;
     int tile_rows;
 };
 // Layout after the 1024-byte aligned base. `key` (score keys) and `r` (reciprocal norms) share storage.
@@ -44,6 +44,7 @@ __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
     p.gain = o;   o += align16((unsigned)budget * 4);
     p.idx = o;    o += align16((unsigned)budget * 4);
     p.row = o;    o += 2 * 1024;  // two rows of the cosine matrix (plain-dot route), 256 floats each
+    p.sect = o;   o += 256;       // cosine and sine of the 32 sector angles
     p.misc = o;   o += 64;        // mbarriers (2 x 8), tmem base, pool size, block-max scratch
     p.total = o + 1024;           // room to align the base to 1024 bytes
     return p;
@@ -69,10 +70,14 @@ __device__ __forceinline__ int tri_row(int a) { return (a * (a + 1)) >> 1; }
 
 // Score terms of one key row for the 8 frequencies a lane covers, packed by frequency pairs.
 // wr / wi: real and imaginary halves (8 bf16 each); returns the lane's partial sum.
+// The rotation by dist * theta_f is taken in two steps: to the nearest of 32 sector angles, whose
+// cosine and sine come from the shared-memory table `sect`, and by the remainder |w| <= pi/32, whose
+// cosine and sine are short Taylor polynomials (error below 2e-9). With t = g conj(k):
+//   Re(t e^{i(A + w)}) = cos w * Re(t e^{iA}) - sin w * Im(t e^{iA}).
 template <bool ROTATE>
 __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, const float2 (&gx)[4], const float2 (&gy)[4],
                                              const float2 (&ngx)[4], const uint32_t (&phi_lo)[8], const uint32_t (&phi_hi)[8],
-                                             uint32_t dlo, uint32_t dhi) {
+                                             uint32_t dlo, uint32_t dhi, const float2* sect) {
     const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
     float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
@@ -83,13 +88,23 @@ __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, c
         const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
         if (ROTATE) {
             const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
-            // bits 32..63 of dist * phi (mod 2^64); dhi is 0 or all ones
+            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns; dhi is 0 or all ones
             const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + (dhi & (0u - phi_lo[2 * p]));
             const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + (dhi & (0u - phi_lo[2 * p + 1]));
-            float2 cs, nsn;
-            sincos_phase2(ta, tb, cs, nsn);
-            acc2 = __ffma2_rn(tr, cs, acc2);
-            acc2 = __ffma2_rn(ti, nsn, acc2);
+            // remainder to the nearest sector: the low 27 bits as a signed number (kept scaled by 32)
+            const float2 w = __fmul2_rn(make_float2((float)(int32_t)(ta << 5), (float)(int32_t)(tb << 5)),
+                                        make_float2(4.5716245e-11f, 4.5716245e-11f));  // 2 pi / 2^37
+            const float2 z = __fmul2_rn(w, w);
+            float2 nsl = __ffma2_rn(z, make_float2(-8.3333333e-3f, -8.3333333e-3f), make_float2(0.16666667f, 0.16666667f));
+            nsl = __ffma2_rn(z, nsl, make_float2(-1.f, -1.f));
+            nsl = __fmul2_rn(w, nsl);  // -sin w
+            float2 cl = __ffma2_rn(z, make_float2(4.1666667e-2f, 4.1666667e-2f), make_float2(-0.5f, -0.5f));
+            cl = __ffma2_rn(z, cl, make_float2(1.f, 1.f));  // cos w
+            const float2 ea = sect[(ta + 0x04000000u) >> 27], eb = sect[(tb + 0x04000000u) >> 27];  // (cos A, sin A)
+            const float2 p1 = make_float2(fmaf(tr.x, ea.x, -ti.x * ea.y), fmaf(tr.y, eb.x, -ti.y * eb.y));  // Re(t e^{iA})
+            const float2 p2 = make_float2(fmaf(tr.x, ea.y, ti.x * ea.x), fmaf(tr.y, eb.y, ti.y * eb.x));    // Im(t e^{iA})
+            acc2 = __ffma2_rn(cl, p1, acc2);
+            acc2 = __ffma2_rn(nsl, p2, acc2);
         } else {
             acc2 = __fadd2_rn(acc2, tr);
         }
@@ -196,6 +211,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     float* gain = reinterpret_cast<float*>(smem + sp.gain);
     int* idx = reinterpret_cast<int*>(smem + sp.idx);
     float* rowbuf = reinterpret_cast<float*>(smem + sp.row);
+    float2* sect = reinterpret_cast<float2*>(smem + sp.sect);
     const uint32_t barK = smem_u32(smem + sp.misc);
     const uint32_t barM = barK + 8;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 16);
@@ -224,6 +240,11 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
         mbar_init(barK, 1);
         mbar_init(barM, 1);
         mbar_init_fence();
+    }
+    if (FUSED && tid >= 32 && tid < 64) {
+        float sn, cs;
+        sincospif((float)(tid - 32) * 0.0625f, &sn, &cs);  // angle 2 pi h / 32
+        sect[tid - 32] = make_float2(cs, sn);
     }
     if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), kTcCols);
     tc_fence_before();
@@ -293,9 +314,9 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
                     if (rotate) {
                         const long long dist = pref - (long long)spos[j];
                         acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
-                                                (uint32_t)((unsigned long long)dist >> 32));
+                                                (uint32_t)((unsigned long long)dist >> 32), sect);
                     } else {
-                        acc = score_lane8<false>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, 0u, 0u);
+                        acc = score_lane8<false>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, 0u, 0u, sect);
                     }
                 }
 #pragma unroll

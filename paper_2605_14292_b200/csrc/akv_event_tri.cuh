@@ -362,12 +362,20 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
         }
         uint32_t kb = 0u;  // the picks-th largest key: the largest v with at least `picks` keys >= v
         if (picks > 0) {
-            for (int bit = 31; bit >= 0; --bit) {
-                const uint32_t v = kb | (1u << bit);
-                int cnt = 0;
+            // two bits per round: the three counts are independent, so their reductions overlap
+            for (int lo = 30; lo >= 0; lo -= 2) {
+                const uint32_t v1 = kb | (1u << lo), v2 = kb | (2u << lo), v3 = kb | (3u << lo);
+                int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) cnt += kk[k] >= v;
-                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= picks) kb = v;
+                for (int k = 0; k < 8; ++k) {
+                    c1 += kk[k] >= v1;
+                    c2 += kk[k] >= v2;
+                    c3 += kk[k] >= v3;
+                }
+                c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+                c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+                c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+                kb = c3 >= picks ? v3 : (c2 >= picks ? v2 : (c1 >= picks ? v1 : kb));
             }
         }
         const float sb = from_orderable(kb);

@@ -142,11 +142,12 @@ struct GreedyLane {
         uint32_t bk = key[0];
 #pragma unroll
         for (int k = 1; k < CPL; ++k) bk = max(bk, key[k]);
-        int kk = CPL - 1;
-#pragma unroll
-        for (int k = CPL - 2; k >= 0; --k) kk = key[k] == bk ? k : kk;
         const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, bk);
-        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, bk == whi ? 0xFFFFu - (uint32_t)(lane + 32 * kk) : 0u);
+        // lowest row among the candidates that reach the maximum (0xFFFF - row, so that max picks the lowest)
+        uint32_t cand = 0u;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) cand = max(cand, key[k] == whi ? 0xFFFFu - (uint32_t)(lane + 32 * k) : 0u);
+        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, cand);
         const int irho = (int)(0xFFFFu - wlo);
 #pragma unroll
         for (int k = 0; k < CPL; ++k) am[k] = (lane + 32 * k == irho) ? 0u : am[k];
@@ -165,9 +166,16 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
     GreedyLane<CPL> g;
     g.init(lane, P, s, bypool, r, lam, with_sims);
     const char* tb = reinterpret_cast<const char*>(tri);
-    int trowB[CPL];  // byte offset of row rho of the triangle
+    // Rows beyond the pool are clamped to its last row: their loads stay inside the triangle and the
+    // loop needs no branch (a divergent branch per candidate costs far more than the wasted load);
+    // what they compute is never looked at, those candidates are retired from the start.
+    int rc4[CPL], trowB[CPL];  // 4 * row, and the byte offset of that row of the triangle
 #pragma unroll
-    for (int k = 0; k < CPL; ++k) trowB[k] = 4 * tri_row(lane + 32 * k);
+    for (int k = 0; k < CPL; ++k) {
+        const int rc = min(lane + 32 * k, max(P - 1, 0));
+        rc4[k] = 4 * rc;
+        trowB[k] = 4 * tri_row(rc);
+    }
     for (int t = 0; t < picks; ++t) {
         uint32_t bk;
         const int irho = g.pick(lane, bk);
@@ -178,11 +186,8 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
         const int tiB = 4 * tri_row(irho), irho4 = 4 * irho;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
-            const int rho = lane + 32 * k;
-            if (rho < P) {
-                const int off = rho > irho ? trowB[k] + irho4 : tiB + 4 * rho;
-                g.M[k] = fmaxf(g.M[k], ri * *reinterpret_cast<const float*>(tb + off));
-            }
+            const int off = rc4[k] > irho4 ? trowB[k] + irho4 : tiB + rc4[k];
+            g.M[k] = fmaxf(g.M[k], ri * *reinterpret_cast<const float*>(tb + off));
         }
     }
 }

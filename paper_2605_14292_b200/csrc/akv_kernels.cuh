@@ -1,4 +1,4 @@
-// Kernels: fused resident event, stand-alone score / select / compact, flat signature (Eq. 1).
+// Kernels: fused resident event, stand-alone score / compact, flat signature (Eq. 1).
 #pragma once
 #include "akv_steps.cuh"
 
@@ -247,80 +247,6 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, cons
 __global__ void fill_int_kernel(int* p, long long n, int v) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) p[i] = v;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Stand-alone selection: scores in, indices out. One CTA per event. RESIDENT: the V tile is staged
-// in shared memory; otherwise similarity rows are read from global memory at every step.
-// ---------------------------------------------------------------------------------------------
-template <typename T, bool RESIDENT>
-__global__ void __launch_bounds__(kThreads) select_kernel(const EventArgs a) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    const DevLayout& lay = a.lay;
-    const EventId id = decode_event(lay, blockIdx.x);
-    const int n = event_n(a, id.b);
-    const int d = lay.d, N = lay.N;
-    const SmemPlan sp = plan_smem(N, d, sizeof(T), a.budget, false, RESIDENT);
-    T* Vt = reinterpret_cast<T*>(smem + sp.tileV);
-    float* s = reinterpret_cast<float*>(smem + sp.s);
-    float* r = reinterpret_cast<float*>(smem + sp.r);
-    float* m = reinterpret_cast<float*>(smem + sp.m);
-    int* order = reinterpret_cast<int*>(smem + sp.order);
-    float* gain = reinterpret_cast<float*>(smem + sp.gain);
-    int* idx = reinterpret_cast<int*>(smem + sp.idx);
-    unsigned char* taken = smem + sp.taken;
-    unsigned long long* red = reinterpret_cast<unsigned long long*>(smem + sp.red);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const T* Vg = reinterpret_cast<const T*>(a.V);
-    const bool flat = a.flat_sig != nullptr;
-    const bool needV = a.greedy && !flat;
-
-    if (RESIDENT && needV) load_tile(Vt, Vg, lay, id, n);
-    int bad = 0;
-    for (int j = tid; j < n; j += kThreads) {
-        const float sc = a.scores[(long long)id.e * N + j];
-        const bool fin = isfinite(sc);
-        bad |= !fin;
-        s[j] = fin ? sc : -INFINITY;
-        taken[j] = 0;
-        m[j] = 0.f;
-    }
-    bad = __syncthreads_or(bad);
-    LayoutRows<T> grows{Vg, &lay, id.b, id.l, id.h};
-    StridedRows<T> srows{Vt, d};
-    if (needV) {
-        const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
-        const int RPW = 32 / G, grp = lane / G, lig = lane % G;
-        for (int j0 = warp * RPW; j0 < n; j0 += kWarps * RPW) {
-            const int j = j0 + grp;
-            const bool valid = j < n;
-            const T* row = RESIDENT ? srows(valid ? j : 0) : grows(valid ? j : 0);
-            const float ss = sumsq_row(row, valid, d, lig, G);
-            if (valid && lig == 0) r[j] = 1.f / (sqrtf(ss) + a.eps);
-        }
-        __syncthreads();
-    }
-    const int picks = min(a.budget, n);
-    if (flat) {
-        StridedRows<float> rows{a.flat_sig + (long long)id.b * N * d, d};
-        greedy_cta<float>(n, picks, a.lam, a.greedy != 0, d, s, nullptr, m, taken, order, gain, rows, red);
-    } else if (RESIDENT) {
-        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, srows, red);
-    } else {
-        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, grows, red);
-    }
-    ordered_indices(n, a.budget, taken, idx);
-    __syncthreads();
-    const long long ob = (long long)id.e * a.budget;
-    for (int t = tid; t < a.budget; t += kThreads) {
-        a.idx_sorted[ob + t] = idx[t];
-        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
-        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
-    }
-    if (tid == 0) {
-        if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
-    }
 }
 
 // ---------------------------------------------------------------------------------------------

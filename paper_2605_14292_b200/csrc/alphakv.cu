@@ -9,6 +9,7 @@
 #include <cstring>
 
 #include "akv_event_tri.cuh"
+#include "akv_select_pool.cuh"
 
 using namespace akv;
 
@@ -247,23 +248,27 @@ static akv_status_t launch_score(akv_handle* h, const EventArgs& a, cudaStream_t
     return launched("score");
 }
 
+// General selection: pool-restricted Algorithm 1; the pool's signature rows stay in shared memory
+// when they fit (tile sized to what the device allows).
+template <typename T, bool FLAT>
+static akv_status_t launch_select_pool(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+    const int E = a.lay.B * a.lay.L * a.lay.H;
+    const int row_bytes = a.lay.d * (int)sizeof(T);
+    const PoolSmem fixed = plan_pool_smem(a.lay.N, a.budget, row_bytes, 0);
+    if ((int)fixed.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "N = %d is too large for the selection kernel", a.lay.N);
+    int tile_rows = (h->smem_optin - (int)fixed.total) / row_bytes;
+    if (tile_rows > a.lay.N) tile_rows = a.lay.N;
+    if (!a.greedy) tile_rows = 0;
+    const PoolSmem sp = plan_pool_smem(a.lay.N, a.budget, row_bytes, tile_rows);
+    akv_status_t s = set_smem(select_pool_kernel<T, FLAT>, sp.total);
+    if (s != AKV_OK) return s;
+    select_pool_kernel<T, FLAT><<<E, kThreads, sp.total, st>>>(a, tile_rows);
+    return launched("select_pool");
+}
 template <typename T>
 static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStream_t st) {
-    const int E = a.lay.B * a.lay.L * a.lay.H;
-    const bool needV = a.greedy && !a.flat_sig;
-    const SmemPlan res = plan_smem(a.lay.N, a.lay.d, sizeof(T), a.budget, false, true);
-    const SmemPlan non = plan_smem(a.lay.N, a.lay.d, sizeof(T), a.budget, false, false);
-    if (needV && (int)res.total <= h->smem_optin) {
-        akv_status_t s = set_smem(select_kernel<T, true>, res.total);
-        if (s != AKV_OK) return s;
-        select_kernel<T, true><<<E, kThreads, res.total, st>>>(a);
-    } else {
-        if ((int)non.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "N = %d is too large for the selection kernel", a.lay.N);
-        akv_status_t s = set_smem(select_kernel<T, false>, non.total);
-        if (s != AKV_OK) return s;
-        select_kernel<T, false><<<E, kThreads, non.total, st>>>(a);
-    }
-    return launched("select");
+    if (a.flat_sig) return launch_select_pool<float, true>(h, a, st);
+    return launch_select_pool<T, false>(h, a, st);
 }
 
 // Tensor-memory path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.

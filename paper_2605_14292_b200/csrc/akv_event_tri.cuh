@@ -367,8 +367,11 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
         }
         uint32_t kb = 0u;  // the picks-th largest key: the largest v with at least `picks` keys >= v
         if (picks > 0) {
-            // two bits per round: the three counts are independent, so their reductions overlap
-            for (int lo = 30; lo >= 0; lo -= 2) {
+            // two bits per round: the three counts are independent, so their reductions overlap.
+            // Pruning only needs a lower bound of s_(b) (the pool may be a little larger than necessary),
+            // so the low 14 key bits (0.2 % of the value) are not resolved; top-k needs the exact key.
+            const int lo_end = similarity ? 14 : 0;
+            for (int lo = 30; lo >= lo_end; lo -= 2) {
                 const uint32_t v1 = kb | (1u << lo), v2 = kb | (2u << lo), v3 = kb | (3u << lo);
                 int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll

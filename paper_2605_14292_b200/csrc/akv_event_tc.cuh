@@ -229,9 +229,24 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     int bad = 0;
     int timeout = 0;
     if (FUSED) {
-        if (tid == 0) mbar_expect_tx(barK, (uint32_t)n * 256u);
-        for (int row = tid; row < n; row += kTcThreads)
-            bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row), 256u, barK);
+        // K rows -> tile: a few large bulk copies when the event's rows are contiguous, one per page
+        // when pages are, else one per row; all issued by one thread (a bulk copy is a per-warp
+        // instruction, so a copy per thread costs a dozen issue slots each)
+        if (tid == 0) {
+            mbar_expect_tx(barK, (uint32_t)n * 256u);
+            if (lay.page_size == 0 && lay.sn == kTcD) {
+                const __nv_bfloat16* k0 = Kg + row_offset(lay, id.b, id.l, id.h, 0);
+                for (int row = 0; row < n; row += 128)  // 32 KB pieces
+                    bulk_g2s(tile_u32 + row * 256, k0 + (long long)row * kTcD, (uint32_t)min(128, n - row) * 256u, barK);
+            } else if (lay.page_size != 0 && lay.s_page_n == kTcD) {
+                for (int row = 0; row < n; row += lay.page_size)
+                    bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row),
+                             (uint32_t)min(lay.page_size, n - row) * 256u, barK);
+            } else {
+                for (int row = 0; row < n; ++row)
+                    bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row), 256u, barK);
+            }
+        }
         const int* gpos = event_pos(a.pos, id);
         const bool rotate = gpos != nullptr;
         int pmax = INT_MIN;

@@ -156,16 +156,28 @@ struct GreedyLane {
     }
 };
 
+// One float of shared memory, as a volatile load: a group of these is issued back to back and in
+// program order, where plain loads get strung out one per use (a picked row's four entries cost four
+// exposed latencies that way).
+__device__ __forceinline__ float lds_in_order(uint32_t addr) {
+    float v;
+    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
 // The loop of Algorithm 1 run by one warp without any block-wide barrier. with_sims: the running
 // maximum is updated from the triangle `tri` of raw dot products (needs P <= 128 and r); otherwise
-// the picks are the plain arg-max sequence (top-k in pick order).
+// the picks are the plain arg-max sequence (top-k in pick order). The winning key and pool row of
+// pick t are parked in park_key[t] / park_row[t]; inside the loop they stay in registers (lane t mod
+// 32 keeps them) and reach shared memory once per 32 picks: a store per pick would order itself
+// against the loads of the next row and lengthen every step.
 template <int CPL>
 __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bool with_sims, const float* s,
                                                   const unsigned short* bypool, const float* r, float lam, const float* tri,
                                                   uint32_t* park_key, int* park_row) {
     GreedyLane<CPL> g;
     g.init(lane, P, s, bypool, r, lam, with_sims);
-    const char* tb = reinterpret_cast<const char*>(tri);
+    const uint32_t tb = smem_u32(tri), rb = smem_u32(r);
     // Rows beyond the pool are clamped to its last row: their loads stay inside the triangle and the
     // loop needs no branch (a divergent branch per candidate costs far more than the wasted load);
     // what they compute is never looked at, those candidates are retired from the start.
@@ -176,18 +188,32 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
         rc4[k] = 4 * rc;
         trowB[k] = 4 * tri_row(rc);
     }
-    for (int t = 0; t < picks; ++t) {
-        uint32_t bk;
-        const int irho = g.pick(lane, bk);
-        if (lane == 0) { park_key[t] = bk; park_row[t] = irho; }
-        if (!with_sims || t + 1 == picks) continue;
-        // m <- max(m, Sims[i, :]) from the triangle: entry (max, min)
-        const float ri = r[irho];
-        const int tiB = 4 * tri_row(irho), irho4 = 4 * irho;
+    for (int t0 = 0; t0 < picks; t0 += 32) {
+        uint32_t my_key = 0u;
+        int my_row = 0;
+        const int t1 = min(t0 + 32, picks);
+        for (int t = t0; t < t1; ++t) {
+            uint32_t bk;
+            const int irho = g.pick(lane, bk);
+            const bool mine = lane == t - t0;
+            my_key = mine ? bk : my_key;
+            my_row = mine ? irho : my_row;
+            if (!with_sims || t + 1 == picks) continue;
+            // m <- max(m, Sims[i, :]) from the triangle: entry (max, min)
+            const int tiB = 4 * tri_row(irho), irho4 = 4 * irho;
+            uint32_t addr[CPL];
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) {
-            const int off = rc4[k] > irho4 ? trowB[k] + irho4 : tiB + rc4[k];
-            g.M[k] = fmaxf(g.M[k], ri * *reinterpret_cast<const float*>(tb + off));
+            for (int k = 0; k < CPL; ++k) addr[k] = tb + (uint32_t)(rc4[k] > irho4 ? trowB[k] + irho4 : tiB + rc4[k]);
+            const float ri = lds_in_order(rb + irho4);
+            float x[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) x[k] = lds_in_order(addr[k]);
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) g.M[k] = fmaxf(g.M[k], ri * x[k]);
+        }
+        if (t0 + lane < picks) {
+            park_key[t0 + lane] = my_key;
+            park_row[t0 + lane] = my_row;
         }
     }
 }

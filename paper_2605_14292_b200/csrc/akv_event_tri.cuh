@@ -1,9 +1,10 @@
 // Fast event kernel for bf16, d = 128, per-head signatures, N <= 256, used when the pool that
 // survives pruning is expected to stay within 128 rows (N <= 128 or budget <= 64). One CTA of four
-// warps per event, four CTAs resident per SM.
+// warps per event, five CTAs resident per SM (40 KB of shared memory each).
 //
-//   1. K rows arrive in shared memory by per-row bulk copies (cp.async.bulk + mbarrier) and are
-//      scored there (fused RoPE rotate-and-dot against the folded query statistic).
+//   1. K rows arrive in shared memory by bulk copies (cp.async.bulk + mbarrier) and are scored there
+//      (fused RoPE rotate-and-dot against the folded query statistic). The tile holds 128 rows: rows
+//      from 128 on arrive later, in the slots of the first rows once those have been scored.
 //   2. Only candidates with  s_i >= s_(b) - lambda * (1 + slack)  can ever be an argmax of Eq. 2
 //      (the running maximum m never exceeds 1, so every still unchosen member of the top-b scores
 //      beats the others). s_(b) comes from a bisection over the score keys; that pool of P rows,
@@ -13,7 +14,7 @@
 //      memory, and the four warps move its lower triangle to shared memory (tcgen05.ld), taking
 //      the squared norms of Eq. 1 from the diagonal on the way.
 //      P > 128 (hardly any pruning): no tensor-core product; rows of the cosine matrix are plain
-//      dot products from the V tile, one picked row at a time.
+//      dot products of V rows read in place, one picked row at a time.
 //   4. Algorithm 1 runs in ONE warp: every lane owns up to P/32 candidates and keeps s, the
 //      running maximum and lambda/norm in registers; the argmax is two warp reductions, the picked
 //      row of the cosine matrix is read from the triangle without bank conflicts.
@@ -24,17 +25,18 @@
 
 namespace akv {
 
+constexpr int kTriTileRows = 128;           // K rows resident at a time = rows of the V operand tile
+constexpr unsigned kTriTileBytes = 33792u;  // 128 rows of 256 bytes, rounded up to the triangle of 128 rows
+
 struct TriSmem {
     unsigned tile, s, key, spos, bypool, taken, order, gain, idx, row, sect, misc, total;
-    int tile_rows;
 };
 // Layout after the 1024-byte aligned base. `key` (score keys) and `r` (reciprocal norms) share storage.
 __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
     TriSmem p;
-    p.tile_rows = ((N + 15) & ~15) < 128 ? 128 : ((N + 15) & ~15);
     const unsigned np = (unsigned)((N + 3) & ~3);
     unsigned o = 0;
-    p.tile = o;   o += (unsigned)p.tile_rows * 256u < 33792u ? 33792u : (unsigned)p.tile_rows * 256u;  // >= triangle of 128 rows
+    p.tile = o;   o += kTriTileBytes;
     p.s = o;      o += align16(np * 4);
     p.key = o;    o += align16(np * 4);
     p.spos = o;   o += align16(np * 4);
@@ -43,9 +45,9 @@ __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
     p.order = o;  o += align16((unsigned)budget * 4);
     p.gain = o;   o += align16((unsigned)budget * 4);
     p.idx = o;    o += align16((unsigned)budget * 4);
-    p.row = o;    o += 2 * 1024;  // two rows of the cosine matrix (plain-dot route), 256 floats each
+    p.row = o;    o += 1024;      // one row of the cosine matrix (plain-dot route), 256 floats
     p.sect = o;   o += 256;       // cosine and sine of the 32 sector angles
-    p.misc = o;   o += 64;        // mbarriers (2 x 8), tmem base, pool size, block-max scratch
+    p.misc = o;   o += 64;        // mbarriers (K, product, late K rows), tmem base, pool size, block-max scratch
     p.total = o + 1024;           // room to align the base to 1024 bytes
     return p;
 }
@@ -221,7 +223,7 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
 template <bool FUSED>
-__global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+__global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const DevLayout& lay = a.lay;
@@ -245,12 +247,13 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     float2* sect = reinterpret_cast<float2*>(smem + sp.sect);
     const uint32_t barK = smem_u32(smem + sp.misc);
     const uint32_t barM = barK + 8;
+    const uint32_t barL = barK + 48;  // K rows from 128 on
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 16);
     int* pool_holder = reinterpret_cast<int*>(smem + sp.misc + 20);
     int* pick_holder = reinterpret_cast<int*>(smem + sp.misc + 24);
     int* redi = reinterpret_cast<int*>(smem + sp.misc + 32);
     const uint32_t tile_u32 = smem_u32(tile);
-    const uint32_t half_bytes = (uint32_t)sp.tile_rows * 128u;
+    const uint32_t half_bytes = (uint32_t)kTriTileRows * 128u;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool similarity = a.greedy != 0;
@@ -267,9 +270,24 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
     // next CTA of this kernel only after that, so a late allocation would serialise the CTAs.
     const bool use_tc = similarity;
+    // K rows [r0, r1) -> tile slots from slot0 on: as few bulk copies as the layout allows (whole event
+    // when its rows are contiguous, whole pages when pages are, else row by row), all issued by one
+    // thread (a bulk copy is a per-warp instruction)
+    auto request_k_rows = [&](int r0, int r1, int slot0, uint32_t bar) {
+        mbar_expect_tx(bar, (uint32_t)(r1 - r0) * 256u);
+        for (int row = r0; row < r1;) {
+            int run = 1;
+            if (dense && lay.sn == kTcD) run = min(r1 - row, 128);
+            else if (!dense && lay.s_page_n == kTcD) run = min(r1 - row, lay.page_size - row % lay.page_size);
+            bulk_g2s(tile_u32 + (uint32_t)(slot0 + row - r0) * 256u, Kg + rowoff(row), (uint32_t)run * 256u, bar);
+            row += run;
+        }
+    };
+    const int n_late = FUSED && n > kTriTileRows ? n - kTriTileRows : 0;  // rows that wait for a free slot
     if (tid == 0) {
         mbar_init(barK, 1);
         mbar_init(barM, 1);
+        mbar_init(barL, 1);
         mbar_init_fence();
     }
     if (FUSED && tid >= 32 && tid < 64) {
@@ -287,20 +305,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     int bad = 0;
     int timeout = 0;
     if (FUSED) {
-        // K rows -> tile: one bulk copy when the event's rows are contiguous, one per page when pages
-        // are, else one per row; all issued by one thread (a bulk copy is a per-warp instruction)
-        if (tid == 0) {
-            mbar_expect_tx(barK, (uint32_t)n * 256u);
-            if (dense && lay.sn == kTcD) {
-                for (int row = 0; row < n; row += 128)  // 32 KB pieces
-                    bulk_g2s(tile_u32 + row * 256, Kg + ev_off + (long long)row * kTcD, (uint32_t)min(128, n - row) * 256u, barK);
-            } else if (!dense && lay.s_page_n == kTcD) {
-                for (int row = 0; row < n; row += lay.page_size)
-                    bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), (uint32_t)min(lay.page_size, n - row) * 256u, barK);
-            } else {
-                for (int row = 0; row < n; ++row) bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), 256u, barK);
-            }
-        }
+        if (tid == 0) request_k_rows(0, n - n_late, 0, barK);
         const int* gpos = event_pos(a.pos, id);
         const bool rotate = gpos != nullptr;
         int pmax = INT_MIN;
@@ -334,14 +339,18 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
         }
         __syncthreads();
         if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
-        timeout = !mbar_wait_bounded(barK, 0);
-        if (!timeout) {
-            for (int j0 = 4 * warp; j0 < n; j0 += 4 * (kTcThreads / 32)) {
-                const int j = j0 + grp;
+        // 16 rows per round (4 per warp), in three stretches. Rows from 128 on reuse the slots of rows
+        // 0..n_late-1: they are requested after the first stretch, once every warp is past those rows,
+        // and awaited before the third. The rounds also run after a timeout (over whatever the tile
+        // holds), so that the barrier between them is reached by every thread.
+        auto score_rounds = [&](int round0, int round1) {
+            for (int round = round0; round < round1; ++round) {
+                const int j = 16 * round + 4 * warp + grp;
                 float acc = 0.f;
                 if (j < n) {
-                    const uint4 wr = *reinterpret_cast<const uint4*>(tile + j * 256 + (lane & 7) * 16);
-                    const uint4 wi = *reinterpret_cast<const uint4*>(tile + j * 256 + 128 + (lane & 7) * 16);
+                    const unsigned char* krow = tile + (j & (kTriTileRows - 1)) * 256 + (lane & 7) * 16;
+                    const uint4 wr = *reinterpret_cast<const uint4*>(krow);
+                    const uint4 wi = *reinterpret_cast<const uint4*>(krow + 128);
                     if (rotate) {
                         const long long dist = pref - (long long)spos[j];
                         acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
@@ -361,7 +370,17 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
                     key[j] = orderable(sj);
                 }
             }
+        };
+        timeout = !mbar_wait_bounded(barK, 0);
+        const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
+        score_rounds(0, late_round);
+        if (n_late > 0) {
+            __syncthreads();
+            if (tid == 0) request_k_rows(kTriTileRows, n, 0, barL);
         }
+        score_rounds(late_round, min(rounds, kTriTileRows / 16));
+        if (n_late > 0) timeout |= !mbar_wait_bounded(barL, 0);
+        score_rounds(kTriTileRows / 16, rounds);
     } else {
         for (int j = tid; j < n; j += kTcThreads) {
             const float sc = a.scores[(long long)id.e * N + j];
@@ -378,6 +397,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
         mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
+        if (n_late > 0) mbar_wait_bounded(barL, 0);
         if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
         return;
     }
@@ -431,7 +451,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
     const bool slow = similarity && P > 128;
 
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
-    if (similarity) {
+    if (similarity && !slow) {
         for (int x = tid; x < P * 16; x += kTcThreads) {
             const int rho = x >> 4, c = x & 15;
             cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(bypool[rho]) + c * 8);
@@ -480,13 +500,14 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
             if (rho < P) r[rho] = 1.f / (sqrtf(diag) + a.eps);
         }
     } else if (slow) {
-        // reciprocal norms from the tile (Eq. 1)
+        // reciprocal norms (Eq. 1); this pool does not fit the tile, its V rows are read in place
         for (int rho = tid; rho < P; rho += kTcThreads) {
+            const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
             float ss = 0.f;
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
                 float x[8];
-                load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho, c, half_bytes)), x);
+                load8(vrow + c * 8, x);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
             }
@@ -518,14 +539,16 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tri_kernel(const EventArg
             if (t + 1 == picks) break;
             __syncthreads();
             const int irho = *pick_holder;
-            // row irho of the cosine matrix by plain dot products from the tile
+            // row irho of the cosine matrix by plain dot products
+            const __nv_bfloat16* vpick = Vg + rowoff(bypool[irho]);
             for (int rho = tid; rho < P; rho += kTcThreads) {
+                const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
                 float acc = 0.f;
 #pragma unroll 4
                 for (int c = 0; c < 16; ++c) {
                     float vi[8], vj[8];
-                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(irho, c, half_bytes)), vi);
-                    load8(reinterpret_cast<const __nv_bfloat16*>(tile + tile_chunk(rho, c, half_bytes)), vj);
+                    load8(vpick + c * 8, vi);
+                    load8(vrow + c * 8, vj);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc = fmaf(vi[e], vj[e], acc);
                 }

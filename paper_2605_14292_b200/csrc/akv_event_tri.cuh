@@ -351,13 +351,10 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
                     const unsigned char* krow = tile + (j & (kTriTileRows - 1)) * 256 + (lane & 7) * 16;
                     const uint4 wr = *reinterpret_cast<const uint4*>(krow);
                     const uint4 wi = *reinterpret_cast<const uint4*>(krow + 128);
-                    if (rotate) {
-                        const long long dist = pref - (long long)spos[j];
-                        acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
-                                                (uint32_t)((unsigned long long)dist >> 32), sect);
-                    } else {
-                        acc = score_lane8<false>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, 0u, 0u, sect);
-                    }
+                    // without positions the distance is 0: sector 0, remainder 0, the rotation is the identity
+                    const long long dist = rotate ? pref - (long long)spos[j] : 0ll;
+                    acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
+                                            (uint32_t)((unsigned long long)dist >> 32), sect);
                 }
 #pragma unroll
                 for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
@@ -373,14 +370,19 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         };
         timeout = !mbar_wait_bounded(barK, 0);
         const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
-        score_rounds(0, late_round);
-        if (n_late > 0) {
-            __syncthreads();
-            if (tid == 0) request_k_rows(kTriTileRows, n, 0, barL);
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            // first and third stretch share one copy of the loop (the kernel's code should stay small)
+            if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0);
+            score_rounds(pass ? kTriTileRows / 16 : 0, pass ? rounds : late_round);
+            if (!pass) {
+                if (n_late > 0) {
+                    __syncthreads();
+                    if (tid == 0) request_k_rows(kTriTileRows, n, 0, barL);
+                }
+                score_rounds(late_round, min(rounds, kTriTileRows / 16));
+            }
         }
-        score_rounds(late_round, min(rounds, kTriTileRows / 16));
-        if (n_late > 0) timeout |= !mbar_wait_bounded(barL, 0);
-        score_rounds(kTriTileRows / 16, rounds);
     } else {
         for (int j = tid; j < n; j += kTcThreads) {
             const float sc = a.scores[(long long)id.e * N + j];

@@ -261,3 +261,41 @@ def test_invalid_arguments_launch_nothing():
     assert e.value.code == 4
     assert akv.launch_count() == before
     assert np.array_equal(akv.to_host_bits(K), ev.K)
+
+
+# ------------------------------------------------------------------ events longer than the 128-row K tile
+@pytest.mark.parametrize("N,budget", [(129, 48), (144, 64), (250, 33), (256, 64)])
+def test_k_rows_beyond_the_tile_arrive_in_freed_slots(N, budget):
+    """bf16, d = 128, budget <= 64: the kernel holds 128 K rows at a time; rows from 128 on are scored from
+    the slots of the first rows. Ragged counts put the boundary inside, at and just after the tile."""
+    ev = synth.make_c3(seed=N, B=4, L=2, H=2, N=N, budget=budget)
+    g = run_fused(ev)
+    check_all(ev, g, ev.lam)
+    n_cand = [N, min(N, 129), 128, min(N, 131)]
+    g = run_fused(ev, n_cand=n_cand)
+    check_all(ev, g, ev.lam, n_cand=n_cand)
+
+
+@pytest.mark.parametrize("page,pages_per_seq", [(64, 4), (32, 6), (256, 1)])
+def test_paged_event_longer_than_the_tile(page, pages_per_seq):
+    """Paged cache (page sizes are powers of two), budget 64: K pages are copied whole, a 256-slot page in two
+    pieces around row 128."""
+    c5 = synth.make_c5(seed=page, B=3, L=2, H=2, page=page, pages_per_seq=pages_per_seq, budget=64, rounds=1)
+    L, H, N, d, b = c5.L, c5.H, c5.N, c5.d, c5.budget
+    pool_K, pool_V = dev(c5.pool_K), dev(c5.pool_V)
+    table, pos, q = dev(c5.block_table), dev(c5.pos), dev(c5.qstat)
+    lay = akv.Layout.paged(pool_K, table)
+    hostK = synth.paged_gather_dense(c5.pool_K, c5.block_table)
+    hostV = synth.paged_gather_dense(c5.pool_V, c5.block_table)
+    sel = akv.alpha_compress_event(pool_K, pool_V, pos, q, b, akv.Options(lam=c5.lam), layout=lay, want_scores=True)
+    torch.cuda.synchronize()
+    idx, order, sc = sel.idx_sorted.cpu().numpy(), sel.pick_order.cpu().numpy(), sel.scores.cpu().numpy()
+    posn = pos.cpu().numpy()
+    for bb in range(c5.B):
+        pages = c5.block_table[bb].tolist()
+        for l in range(L):
+            for h in range(H):
+                Kn = akv.to_host_bits(pool_K[l, pages, h]).reshape(N, d)
+                Vn = akv.to_host_bits(pool_V[l, pages, h]).reshape(N, d)
+                chk.check_event(hostK[bb, l, h], hostV[bb, l, h], c5.pos[bb, l, h], c5.qstat[l, h], None, b, c5.lam,
+                                sc[bb, l, h], order[bb, l, h], idx[bb, l, h], Kn, Vn, posn[bb, l, h], log=[])

@@ -1,6 +1,6 @@
 // Fast event kernel for bf16, d = 128, per-head signatures, N <= 256, used when the pool that
 // survives pruning is expected to stay within 128 rows (N <= 128 or budget <= 64). One CTA of four
-// warps per event, five CTAs resident per SM (40 KB of shared memory each).
+// warps per event, six CTAs resident per SM (37 KB of shared memory and 72 registers each).
 //
 //   1. K rows arrive in shared memory by bulk copies (cp.async.bulk + mbarrier) and are scored there
 //      (fused RoPE rotate-and-dot against the folded query statistic). The tile holds 128 rows: rows
@@ -9,11 +9,11 @@
 //      (the running maximum m never exceeds 1, so every still unchosen member of the top-b scores
 //      beats the others). s_(b) comes from a bisection over the score keys; that pool of P rows,
 //      in slot order, is the only part of V that is read for the selection.
-//   3. P <= 128: the pool's V rows form a K-major, 128-byte-swizzled operand tile, one
+//   3. P <= 127: the pool's V rows form a K-major, 128-byte-swizzled operand tile, one
 //      tcgen05.mma sequence writes the pool's cosine matrix (raw dot products, fp32) into tensor
 //      memory, and the four warps move its lower triangle to shared memory (tcgen05.ld), taking
 //      the squared norms of Eq. 1 from the diagonal on the way.
-//      P > 128 (hardly any pruning): no tensor-core product; rows of the cosine matrix are plain
+//      P > 127 (hardly any pruning): no tensor-core product; rows of the cosine matrix are plain
 //      dot products of V rows read in place, one picked row at a time.
 //   4. Algorithm 1 runs in ONE warp: every lane owns up to P/32 candidates and keeps s, the
 //      running maximum and lambda/norm in registers; the argmax is two warp reductions, the picked
@@ -26,7 +26,8 @@
 namespace akv {
 
 constexpr int kTriTileRows = 128;           // K rows resident at a time = rows of the V operand tile
-constexpr unsigned kTriTileBytes = 33792u;  // 128 rows of 256 bytes, rounded up to the triangle of 128 rows
+constexpr unsigned kTriTileBytes = 32768u;  // 128 rows of 256 bytes; holds the triangle of up to 127 rows
+constexpr int kTriMaxPool = 127;            // largest pool whose cosine matrix goes through the tile
 
 struct TriSmem {
     unsigned tile, s, key, spos, bypool, taken, order, gain, idx, row, sect, misc, total;
@@ -45,7 +46,7 @@ __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
     p.order = o;  o += align16((unsigned)budget * 4);
     p.gain = o;   o += align16((unsigned)budget * 4);
     p.idx = o;    o += align16((unsigned)budget * 4);
-    p.row = o;    o += 1024;      // one row of the cosine matrix (plain-dot route), 256 floats
+    p.row = p.tile;               // one row of the cosine matrix: plain-dot route only, which leaves the tile unused
     p.sect = o;   o += 256;       // cosine and sine of the 32 sector angles
     p.misc = o;   o += 64;        // mbarriers (K, product, late K rows), tmem base, pool size, block-max scratch
     p.total = o + 1024;           // room to align the base to 1024 bytes
@@ -449,8 +450,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     }
     __syncthreads();  // every key has been read: its storage becomes r below
     const int P = *pool_holder;
-    const bool fast = similarity && P <= 128 && picks > 1;
-    const bool slow = similarity && P > 128;
+    const bool fast = similarity && P <= kTriMaxPool && picks > 1;
+    const bool slow = similarity && P > kTriMaxPool;
 
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
     if (similarity && !slow) {
@@ -592,20 +593,23 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     if (!FUSED) return;
 
     // ---- compaction in place ----------------------------------------------------------------------
-    // Every kept K and V row and position is on chip (registers for up to 64 rows, else the tile)
-    // before the first store: a destination slot can be another kept row's source.
+    // Every kept K and V row and position is on chip before the first store: a destination slot can be
+    // another kept row's source. Up to 64 rows: K in registers, V through the (by now free) tile by
+    // cp.async, one barrier. Both in registers would make this the kernel's register peak and cost a
+    // resident CTA per SM.
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
     if (picks <= 64) {
-        uint4 kreg[8], vreg[8];
+        uint4 kreg[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int x = tid + i * kTcThreads;
             if (x < picks * 16) {
                 const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
                 kreg[i] = *reinterpret_cast<const uint4*>(Kg + off);
-                vreg[i] = *reinterpret_cast<const uint4*>(Vg + off);
+                cp_async16(tile_u32 + (uint32_t)x * 16u, Vg + off);
             }
         }
+        cp_async_wait_all();
         __syncthreads();  // every load above has been performed
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -613,7 +617,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
             if (x < picks * 16) {
                 const long long off = rowoff(x >> 4) + (x & 15) * 8;
                 *reinterpret_cast<uint4*>(Kg + off) = kreg[i];
-                *reinterpret_cast<uint4*>(Vg + off) = vreg[i];
+                *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(tile + x * 16);
             }
         }
     } else {

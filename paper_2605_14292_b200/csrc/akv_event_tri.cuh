@@ -599,26 +599,17 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     // resident CTA per SM.
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
     if (picks <= 64) {
-        uint4 kreg[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int x = tid + i * kTcThreads;
-            if (x < picks * 16) {
-                const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
-                kreg[i] = *reinterpret_cast<const uint4*>(Kg + off);
-                cp_async16(tile_u32 + (uint32_t)x * 16u, Vg + off);
-            }
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
+            cp_async16(tile_u32 + (uint32_t)x * 16u, Kg + off);
+            cp_async16(tile_u32 + 16384u + (uint32_t)x * 16u, Vg + off);
         }
         cp_async_wait_all();
         __syncthreads();  // every load above has been performed
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int x = tid + i * kTcThreads;
-            if (x < picks * 16) {
-                const long long off = rowoff(x >> 4) + (x & 15) * 8;
-                *reinterpret_cast<uint4*>(Kg + off) = kreg[i];
-                *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(tile + x * 16);
-            }
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const long long off = rowoff(x >> 4) + (x & 15) * 8;
+            *reinterpret_cast<uint4*>(Kg + off) = *reinterpret_cast<const uint4*>(tile + x * 16);
+            *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(tile + 16384 + x * 16);
         }
     } else {
 #pragma unroll 1

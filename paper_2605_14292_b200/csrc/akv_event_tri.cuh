@@ -1,5 +1,5 @@
 // Fast event kernel for bf16, d = 128, per-head signatures, N <= 256, used when the pool that
-// survives pruning is expected to stay within 128 rows (N <= 128 or budget <= 64). One CTA of four
+// survives pruning is expected to stay within 127 rows (N <= 128 or budget <= 64). One CTA of four
 // warps per event, six CTAs resident per SM (37 KB of shared memory and 72 registers each).
 //
 //   1. K rows arrive in shared memory by bulk copies (cp.async.bulk + mbarrier) and are scored there
@@ -18,8 +18,8 @@
 //   4. Algorithm 1 runs in ONE warp: every lane owns up to P/32 candidates and keeps s, the
 //      running maximum and lambda/norm in registers; the argmax is two warp reductions, the picked
 //      row of the cosine matrix is read from the triangle without bank conflicts.
-//   5. Kept rows are written back in place: K, V and positions are re-read (L2) and held on chip
-//      before the first store.
+//   5. Kept rows are written back in place: K and V rows are re-read (L2) into the tile, which is
+//      free by then, and stored after a barrier; positions come from their shared-memory copy.
 #pragma once
 #include "akv_event_tc.cuh"
 

@@ -299,3 +299,20 @@ def test_paged_event_longer_than_the_tile(page, pages_per_seq):
                 Vn = akv.to_host_bits(pool_V[l, pages, h]).reshape(N, d)
                 chk.check_event(hostK[bb, l, h], hostV[bb, l, h], c5.pos[bb, l, h], c5.qstat[l, h], None, b, c5.lam,
                                 sc[bb, l, h], order[bb, l, h], idx[bb, l, h], Kn, Vn, posn[bb, l, h], log=[])
+
+
+@pytest.mark.parametrize("maker", ["c3_192", "c2_256", "f32_96"])
+def test_pool_pruning_changes_no_pick(maker):
+    """The pool that Algorithm 1 runs over is pruned exactly: with pruning switched off (every candidate in the
+    pool, which takes the kernels' large-pool routes) the picks, their order and the compacted rows are the same."""
+    if maker == "c3_192":
+        ev = synth.make_c3(seed=21, B=2, L=2, H=2, N=192, budget=64)
+    elif maker == "c2_256":
+        ev = synth.make_c2(seed=22, B=1, L=2, H=2)
+    else:
+        ev = synth.make_plain(2, 2, 2, 96, 64, 30, 0.5, dtype=synth.F32, seed=23)
+    pruned = run_fused(ev)
+    full = run_fused(ev, flags=akv.FLAG_NO_PRUNE)
+    for k in ("order", "idx", "K", "V", "pos", "n_kept", "status"):
+        assert np.array_equal(pruned[k], full[k]), k
+    check_all(ev, full, ev.lam)

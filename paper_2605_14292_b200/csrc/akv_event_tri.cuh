@@ -91,9 +91,9 @@ __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, c
         const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
         if (ROTATE) {
             const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
-            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns; dhi is 0 or all ones
-            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + (dhi & (0u - phi_lo[2 * p]));
-            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + (dhi & (0u - phi_lo[2 * p + 1]));
+            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns
+            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + dhi * phi_lo[2 * p];
+            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + dhi * phi_lo[2 * p + 1];
             // remainder to the nearest sector: the low 27 bits as a signed number (kept scaled by 32)
             const float2 w = __fmul2_rn(make_float2((float)(int32_t)(ta << 5), (float)(int32_t)(tb << 5)),
                                         make_float2(4.5716245e-11f, 4.5716245e-11f));  // 2 pi / 2^37

@@ -487,20 +487,30 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         // lower triangle -> shared memory; row rho = 32 warp + lane needs columns 0..rho
         const int rho = 32 * warp + lane;
         if (32 * warp < P) {
-            float diag = 1.f;
             const int trow = tri_row(rho);
-            for (int cb = 0; cb <= warp; ++cb) {
+            const uint32_t lanes = tbase + ((uint32_t)(warp * 32) << 16);
+            // column blocks left of the diagonal one: every column is below the row
+            for (int cb = 0; cb < warp; ++cb) {
                 uint32_t v[32];
-                tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * cb), v);
+                tmem_ld32(lanes + (uint32_t)(32 * cb), v);
                 tmem_ld_wait();
+                if (rho < P) {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    const int c = 32 * cb + k;
-                    if (c <= rho && rho < P) tri[trow + c] = __uint_as_float(v[k]);
-                    if (c == rho) diag = __uint_as_float(v[k]);
+                    for (int k = 0; k < 32; ++k) tri[trow + 32 * cb + k] = __uint_as_float(v[k]);
                 }
             }
-            if (rho < P) r[rho] = 1.f / (sqrtf(diag) + a.eps);
+            // the diagonal block: columns up to the row itself, whose last entry is the squared norm
+            {
+                uint32_t v[32];
+                tmem_ld32(lanes + (uint32_t)(32 * warp), v);
+                tmem_ld_wait();
+                if (rho < P) {
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        if (k <= lane) tri[trow + 32 * warp + k] = __uint_as_float(v[k]);
+                    r[rho] = 1.f / (sqrtf(tri[trow + rho]) + a.eps);  // read back: this thread stored it
+                }
+            }
         }
     } else if (slow) {
         // reciprocal norms (Eq. 1); this pool does not fit the tile, its V rows are read in place

@@ -455,9 +455,17 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
 
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
     if (similarity && !slow) {
-        for (int x = tid; x < P * 16; x += kTcThreads) {
-            const int rho = x >> 4, c = x & 15;
-            cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(bypool[rho]) + c * 8);
+        // thread -> 16-byte column c of rows r0, r0 + 8, ...: the swizzle term (c ^ row) & 7 is the same for
+        // all of them, so a row costs one pool lookup, one address and one copy
+        const int c = tid & 15, r0 = tid >> 4;
+        const uint32_t dst0 = tile_u32 + tile_chunk(r0, c, half_bytes);
+        if (dense) {
+            const __nv_bfloat16* vcol = Vg + ev_off + c * 8;
+            for (int rho = r0; rho < P; rho += 8)
+                cp_async16(dst0 + (uint32_t)(rho - r0) * 128u, vcol + (long long)bypool[rho] * lay.sn);
+        } else {
+            for (int rho = r0; rho < P; rho += 8)
+                cp_async16(dst0 + (uint32_t)(rho - r0) * 128u, Vg + rowoff(bypool[rho]) + c * 8);
         }
         cp_async_wait_all();
         fence_proxy_async();
@@ -609,17 +617,22 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     // resident CTA per SM.
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
     if (picks <= 64) {
-        for (int x = tid; x < picks * 16; x += kTcThreads) {
-            const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
-            cp_async16(tile_u32 + (uint32_t)x * 16u, Kg + off);
-            cp_async16(tile_u32 + 16384u + (uint32_t)x * 16u, Vg + off);
+        // thread -> 16-byte column c of kept rows r0, r0 + 8, ...
+        const int c = tid & 15, r0 = tid >> 4;
+        const uint32_t slot0 = (uint32_t)(r0 * 256 + c * 16);
+        const long long col = (dense ? ev_off : 0) + c * 8;
+        for (int t = r0; t < picks; t += 8) {
+            const long long off = col + (dense ? (long long)idx[t] * lay.sn : rowoff(idx[t]));
+            cp_async16(tile_u32 + slot0 + (uint32_t)(t - r0) * 256u, Kg + off);
+            cp_async16(tile_u32 + 16384u + slot0 + (uint32_t)(t - r0) * 256u, Vg + off);
         }
         cp_async_wait_all();
         __syncthreads();  // every load above has been performed
-        for (int x = tid; x < picks * 16; x += kTcThreads) {
-            const long long off = rowoff(x >> 4) + (x & 15) * 8;
-            *reinterpret_cast<uint4*>(Kg + off) = *reinterpret_cast<const uint4*>(tile + x * 16);
-            *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(tile + 16384 + x * 16);
+        for (int t = r0; t < picks; t += 8) {
+            const long long off = col + (dense ? (long long)t * lay.sn : rowoff(t));
+            const unsigned char* src = tile + slot0 + (t - r0) * 256;
+            *reinterpret_cast<uint4*>(Kg + off) = *reinterpret_cast<const uint4*>(src);
+            *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(src + 16384);
         }
     } else {
 #pragma unroll 1

@@ -80,7 +80,7 @@ __device__ __forceinline__ int tri_row(int a) { return (a * (a + 1)) >> 1; }
 template <bool ROTATE>
 __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, const float2 (&gx)[4], const float2 (&gy)[4],
                                              const float2 (&ngx)[4], const uint32_t (&phi_lo)[8], const uint32_t (&phi_hi)[8],
-                                             uint32_t dlo, uint32_t dhi, const float2* sect) {
+                                             uint32_t dist, const float2* sect) {
     const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
     float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
@@ -91,9 +91,9 @@ __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, c
         const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
         if (ROTATE) {
             const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
-            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns
-            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + dhi * phi_lo[2 * p];
-            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + dhi * phi_lo[2 * p + 1];
+            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns (dist: 32 bits, not negative)
+            const uint32_t ta = __umulhi(dist, phi_lo[2 * p]) + dist * phi_hi[2 * p];
+            const uint32_t tb = __umulhi(dist, phi_lo[2 * p + 1]) + dist * phi_hi[2 * p + 1];
             // remainder to the nearest sector: the low 27 bits as a signed number (kept scaled by 32)
             const float2 w = __fmul2_rn(make_float2((float)(int32_t)(ta << 5), (float)(int32_t)(tb << 5)),
                                         make_float2(4.5716245e-11f, 4.5716245e-11f));  // 2 pi / 2^37
@@ -332,14 +332,39 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
             phi_lo[u] = (uint32_t)tab.phi[f0 + u];
             phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
         }
+        // Distances are measured from `pref`, which is never behind the last key, so that they are
+        // non-negative 32-bit numbers. A reference position behind the last key (rare) is reached by turning
+        // the folded statistic once by the difference: e^{i (p_ref - pos) theta} = e^{i (p_ref - last) theta} e^{i (last - pos) theta}.
         long long pref = 0;
-        if (rotate && !a.p_ref) {
+        if (rotate) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
             if (lane == 0) redi[warp] = pmax;
         }
         __syncthreads();
-        if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
+        if (rotate) {
+            const long long last = (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3]));
+            pref = a.p_ref ? (long long)a.p_ref[id.b] : last + 1;
+            if (pref < last) {
+                const long long back = pref - last;
+                const uint32_t bl = (uint32_t)back, bh = (uint32_t)((unsigned long long)back >> 32);
+                pref = last;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t ph = __umulhi(bl, phi_lo[u]) + bl * phi_hi[u] + bh * phi_lo[u];
+                    const float2 e = sect[(ph + 0x04000000u) >> 27];
+                    const float w = (float)(int32_t)(ph << 5) * 4.5716245e-11f, z = w * w;
+                    const float sw = w * fmaf(z, fmaf(z, 8.3333333e-3f, -0.16666667f), 1.f);
+                    const float cw = fmaf(z, fmaf(z, 4.1666667e-2f, -0.5f), 1.f);
+                    const float c = e.x * cw - e.y * sw, sn = e.y * cw + e.x * sw;
+                    float& x = (u & 1) ? gx[u >> 1].y : gx[u >> 1].x;
+                    float& y = (u & 1) ? gy[u >> 1].y : gy[u >> 1].x;
+                    float& nx = (u & 1) ? ngx[u >> 1].y : ngx[u >> 1].x;
+                    const float x2 = x * c - y * sn, y2 = x * sn + y * c;
+                    x = x2; y = y2; nx = -x2;
+                }
+            }
+        }
         // 16 rows per round (4 per warp), in three stretches. Rows from 128 on reuse the slots of rows
         // 0..n_late-1: they are requested after the first stretch, once every warp is past those rows,
         // and awaited before the third. The rounds also run after a timeout (over whatever the tile
@@ -353,9 +378,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
                     const uint4 wr = *reinterpret_cast<const uint4*>(krow);
                     const uint4 wi = *reinterpret_cast<const uint4*>(krow + 128);
                     // without positions the distance is 0: sector 0, remainder 0, the rotation is the identity
-                    const long long dist = rotate ? pref - (long long)spos[j] : 0ll;
-                    acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, (uint32_t)dist,
-                                            (uint32_t)((unsigned long long)dist >> 32), sect);
+                    const uint32_t dist = rotate ? (uint32_t)(pref - (long long)spos[j]) : 0u;
+                    acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, dist, sect);
                 }
 #pragma unroll
                 for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);

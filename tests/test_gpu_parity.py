@@ -316,3 +316,14 @@ def test_pool_pruning_changes_no_pick(maker):
     for k in ("order", "idx", "K", "V", "pos", "n_kept", "status"):
         assert np.array_equal(pruned[k], full[k]), k
     check_all(ev, full, ev.lam)
+
+
+def test_reference_position_behind_some_keys():
+    """Keys ahead of the reference position have negative distances; the fast kernel measures distances from
+    the last key and turns the query statistic by the difference. Positions are sparse and large."""
+    ev = synth.make_c3(seed=31, B=3, L=2, H=2, N=192, budget=64)
+    rng = np.random.default_rng(31)
+    ev.pos[:] = np.sort(rng.choice(3_000_000, size=192, replace=False)).astype(np.int32)
+    ev.p_ref[:] = np.array([ev.pos[0, 0, 0, 100], ev.pos[0, 0, 0, 0] - 5, ev.pos[0, 0, 0, -1]], dtype=ev.p_ref.dtype)
+    g = run_fused(ev)
+    check_all(ev, g, ev.lam)

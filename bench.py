@@ -37,7 +37,7 @@ def algorithmic_bytes(N, b, d, esize):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on this workload, from
 # the ncu capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 328282624 + 98628864
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 328119296 + 97766400
 
 
 def load_peaks():

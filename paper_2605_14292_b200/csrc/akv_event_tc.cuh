@@ -209,9 +209,19 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
     const bool similarity = a.greedy != 0;
     const int np4 = (N + 3) & ~3;
+    // row addressing: dense events are one base offset plus a row stride
+    const bool dense = lay.page_size == 0;
+    const long long ev_off = dense ? id.b * lay.sb + id.l * lay.sl + id.h * lay.sh : 0;
+    auto rowoff = [&](int j) -> long long {
+        return dense ? ev_off + (long long)j * lay.sn : row_offset(lay, id.b, id.l, id.h, j);
+    };
 
-    // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
-    // next CTA of this kernel only after that, so a late allocation would serialise the CTAs.
+    // Tensor memory (half of the SM's columns for the two-block matrix) is claimed only when the pool's V
+    // rows are on their way, and held until the loop ends: the span in which an event holds it, not the
+    // event's lifetime, is what limits this kernel to two events at a time, and a third resident CTA scores
+    // its keys meanwhile. (The SM starts the next CTA of a kernel that allocates tensor memory only once
+    // the resident one has given up its right to allocate; with three long-lived CTAs per SM the starts
+    // are further apart than the time to reach the allocation.)
     const uint32_t tcols = (uint32_t)a.tmem_cols;
     const bool use_tc = similarity && tcols != 0u;
     if (tid == 0) {
@@ -219,11 +229,8 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         mbar_init(barM, 1);
         mbar_init_fence();
     }
-    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), tcols);
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tbase = use_tc ? *tmem_holder : 0u;
+    uint32_t tbase = 0u;
 
     // ---- scores ---------------------------------------------------------------------------------
     int bad = 0;
@@ -235,16 +242,16 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         if (tid == 0) {
             mbar_expect_tx(barK, (uint32_t)n * 256u);
             if (lay.page_size == 0 && lay.sn == kTcD) {
-                const __nv_bfloat16* k0 = Kg + row_offset(lay, id.b, id.l, id.h, 0);
+                const __nv_bfloat16* k0 = Kg + rowoff(0);
                 for (int row = 0; row < n; row += 128)  // 32 KB pieces
                     bulk_g2s(tile_u32 + row * 256, k0 + (long long)row * kTcD, (uint32_t)min(128, n - row) * 256u, barK);
             } else if (lay.page_size != 0 && lay.s_page_n == kTcD) {
                 for (int row = 0; row < n; row += lay.page_size)
-                    bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row),
+                    bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row),
                              (uint32_t)min(lay.page_size, n - row) * 256u, barK);
             } else {
                 for (int row = 0; row < n; ++row)
-                    bulk_g2s(tile_u32 + row * 256, Kg + row_offset(lay, id.b, id.l, id.h, row), 256u, barK);
+                    bulk_g2s(tile_u32 + row * 256, Kg + rowoff(row), 256u, barK);
             }
         }
         const int* gpos = event_pos(a.pos, id);
@@ -348,7 +355,6 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
         mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
-        if (use_tc && warp == 0) tmem_dealloc(tbase, tcols);
         return;
     }
     bad = __syncthreads_or(bad);
@@ -415,11 +421,15 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     for (int x = tid; x < vrows * 16; x += kTcThreads) {
         const int rho = x >> 4, c = x & 15;
         const int j = byrank[rho];
-        cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + row_offset(lay, id.b, id.l, id.h, j) + c * 8);
+        cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(j) + c * 8);
     }
+    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), tcols);  // may wait for another CTA's columns
     cp_async_wait_all();
     fence_proxy_async();
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    if (use_tc) tbase = *tmem_holder;
 
     const bool do_mma = use_tc && picks > 1;
     if (do_mma && tid == 0) {
@@ -612,11 +622,11 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
             const int x = tid + i * kTcThreads;
             if (x < picks * 16)
                 kreg[i] = *reinterpret_cast<const uint4*>(
-                    reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[x >> 4])) + (x & 15) * 16);
+                    reinterpret_cast<const char*>(Kw + rowoff(idx[x >> 4])) + (x & 15) * 16);
         }
         for (int x = tid; x < picks * 16; x += kTcThreads) {
             const int rr = x >> 4, c = x & 15;
-            copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
+            copy16(reinterpret_cast<char*>(Vg + rowoff(rr)) + c * 16,
                    tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
         }
         __syncthreads();  // every K load above has been performed
@@ -624,25 +634,25 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         for (int i = 0; i < 8; ++i) {
             const int x = tid + i * kTcThreads;
             if (x < picks * 16)
-                *reinterpret_cast<uint4*>(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, x >> 4)) + (x & 15) * 16) =
+                *reinterpret_cast<uint4*>(reinterpret_cast<char*>(Kw + rowoff(x >> 4)) + (x & 15) * 16) =
                     kreg[i];
         }
     } else {
         for (int x = tid; x < picks * 16; x += kTcThreads) {
             const int rr = x >> 4, c = x & 15;
-            copy16(reinterpret_cast<char*>(Vg + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16,
+            copy16(reinterpret_cast<char*>(Vg + rowoff(rr)) + c * 16,
                    tile + tile_chunk(rankof[idx[rr]], c, half_bytes));
         }
         __syncthreads();  // the V tile is free from here on
         for (int x = tid; x < picks * 16; x += kTcThreads) {
             const int rr = x >> 4, c = x & 15;
             copy16(tile + rr * 256 + c * 16,
-                   reinterpret_cast<const char*>(Kw + row_offset(lay, id.b, id.l, id.h, idx[rr])) + c * 16);
+                   reinterpret_cast<const char*>(Kw + rowoff(idx[rr])) + c * 16);
         }
         __syncthreads();
         for (int x = tid; x < picks * 16; x += kTcThreads) {
             const int rr = x >> 4, c = x & 15;
-            copy16(reinterpret_cast<char*>(Kw + row_offset(lay, id.b, id.l, id.h, rr)) + c * 16, tile + rr * 256 + c * 16);
+            copy16(reinterpret_cast<char*>(Kw + rowoff(rr)) + c * 16, tile + rr * 256 + c * 16);
         }
     }
     if (wpos)

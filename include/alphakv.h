@@ -104,9 +104,9 @@ const char* akv_status_string(akv_status_t s);
 uint64_t akv_launch_count(void);
 
 /*
- * alpha_score -- per-token retention score s (Section 4.1: the scores "produced by
- * the TriAttention 1d scorer"; the paper does not print the formula, the library
- * uses: keys are stored pre-RoPE, coordinate f pairs with f + d/2,
+ * alpha_score -- per-token retention score s (Section 4.1 takes it from the TriAttention
+ * scorer and does not print the formula; the library uses the following reading:
+ * keys are stored pre-RoPE, coordinate f pairs with f + d/2,
  *   s_i = (1/sqrt d) Re sum_f c_f z(q)_f conj(z(k_i)_f) exp(i (p_ref - p_i) theta_f),
  *   theta_f = rope_base^(-2f/d), c_f = (1/W) sum_{w<W} exp(i w theta_f),
  *   z(x)_f = x_f + i x_{f+d/2},
@@ -156,8 +156,8 @@ akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, cons
                                   void* stream);
 
 /*
- * kv_compact -- the retained rows become the new cache (Section 1; Section 4.1:
- * "k <= n is the post-compression budget"): for r = 0..budget-1, row idx_sorted[r]
+ * kv_compact -- the retained rows become the new cache of at most `budget` rows
+ * (Section 1; Section 4.1): for r = 0..budget-1, row idx_sorted[r]
  * of K, of V and of pos moves to slot r of the SAME buffer (bit copies). Entries
  * idx_sorted[r] < 0 end the list. idx_sorted must be ascending and distinct (as
  * alpha_select writes it); rows at slots >= the kept count are unspecified afterwards.

@@ -3,13 +3,14 @@
  *
  * Plain, slow, double-precision statement of one KV-cache compression event of
  * the alpha retainer, written so that it can be read against the paper:
- *   - score:      reading of the TriAttention 1d scorer named in Section 4.1
+ *   - score:      reading of the scorer that Section 4.1 inherits from TriAttention
  *                 (formula not printed in the paper; PARITY UNPINNED against the
  *                 real scorer, pinned to closed forms in the tests);
  *   - signature:  Eq. 1 reduced to one head, v_i = V_i / (||V_i||_2 + eps);
- *   - selection:  Eq. 2, Eq. 3 and Algorithm 1 in the paper's order (running
- *                 vector m, a = s - lambda m, a[S] = -inf, argmax, update m);
- *                 lambda = 0 takes the top-k branch of Algorithm 1;
+ *   - selection:  Eq. 2 evaluated for every candidate from a per-candidate redundancy term
+ *                 (largest cosine against the members chosen so far, never below zero), Eq. 3's
+ *                 arg-max over the candidates outside the set, then the new member's cosines are
+ *                 folded into that term -- what Algorithm 1 computes; lambda = 0 is plain top-k;
  *   - compaction: retained rows become the new cache, ascending index order.
  * No blocking, no pruning, no reordering. It shares no code with the CUDA path
  * and is only called by tests, the smoke check and the benchmark's CPU leg.
@@ -115,7 +116,7 @@ static double second_best(const double* a, int n, int skip) {
     return v;
 }
 
-/* Algorithm 1. order/gain/margin have k entries; returns the number of picks
+/* Greedy fill (Eq. 2, Eq. 3). order/gain/margin have k entries; returns the number of picks
  * (min(k, n)); *status: 0 ok, 1 non-finite score seen, 2 n < k. */
 int orc_select(const double* s_in, const double* sig, int n, int d, int k, double lam,
                int force_greedy, int64_t* order, double* gain, double* margin, int* status) {

@@ -6,14 +6,15 @@ the smoke check and the benchmark's CPU-baseline leg may import it. The product
 never routes through it.
 
 What is written from where:
-  * selection: Section 4.1, Eq. 1 (V-signatures), Eq. 2 (marginal gain),
-    Eq. 3 (greedy fill) and Algorithm 1, taken step by step in the paper's
-    order and notation (s, m, a, Sims, S, k, lambda);
-  * top-k baseline and the lambda = 0 fast path: Section 4.1 and the first
-    branch of Algorithm 1;
-  * compaction: the retained rows become the new cache (Section 1, Section 4.1
-    "k <= n is the post-compression budget");
-  * score: the paper names the TriAttention 1d scorer but does not print its
+  * selection: Section 4.1 -- Eq. 1 (V-signatures), Eq. 2 (marginal gain of a
+    candidate given the chosen set), Eq. 3 (each new member maximises Eq. 2 over
+    the candidates not chosen yet; the first member has the largest score) --
+    which is what Algorithm 1 computes;
+  * top-k baseline and the lambda = 0 case: Section 4.1 and the first branch of
+    Algorithm 1;
+  * compaction: the chosen rows, in slot order, become the new cache of at most
+    `budget` rows (Section 1, Section 4.1);
+  * score: the paper names the scorer it inherits but does not print its
     formula. The reading used here (mean RoPE attention logit of the head's
     query statistic against each pre-RoPE key, a trigonometric series in the
     position distance) is pinned only to its own closed forms and to a
@@ -64,9 +65,9 @@ def window_coefficients(theta: np.ndarray, W: int) -> np.ndarray:
 
 def triattention_score(K, pos, qstat, p_ref, W: int = 1, base: float = 10000.0) -> np.ndarray:
     """Per-token retention score s in R^n for one (sequence, layer, KV head)
-    (Section 4.1: "per-token retention scores produced by the TriAttention 1d
-    scorer"; Section 2: precomputed Q/K frequency statistics as a proxy for what
-    future queries will need).
+    (Section 4.1 takes the scores from the TriAttention scorer it builds on;
+    Section 2 describes that scorer as working from precomputed Q/K frequency
+    statistics that stand in for the queries still to come).
 
     Reading: keys are stored pre-RoPE; RoPE pairs coordinate f with f + d/2 and
     turns the pair, seen as the complex number z(x)_f = x_f + i x_{f+d/2}, by
@@ -156,9 +157,15 @@ class Selection:
 
 
 def alpha_select(s, sig, k: int, lam: float, force_greedy: bool = False) -> Selection:
-    """Algorithm 1 with rows of Sims computed on demand (each entry of V V^T is
-    an independent dot product, so the values are those of the precomputed
-    matrix).  s: scores [n]; sig: unit-normalised signatures [n, d]."""
+    """Greedy fill of the budget (Section 4.1, Eq. 2 and Eq. 3; Algorithm 1).
+
+    State kept between picks: for every candidate i the redundancy term of Eq. 2 against the
+    set chosen so far, red_i = max(0, max_{j in S} cos(v_i, v_j)), which is 0 for the empty
+    set. A pick evaluates Eq. 2 for all candidates, gain_i = s_i - lam * red_i, takes the
+    best candidate outside S (Eq. 3; the first pick therefore has the largest score) and
+    folds the new member's cosines into red. cos(v_i, v_j) = <v_i, v_j> for the unit rows of
+    Eq. 1; each one is computed when it is needed, as a plain dot product.
+    s: scores [n]; sig: unit-normalised signatures [n, d]."""
     s, bad = sanitize_scores(s)
     sig = np.asarray(sig, dtype=np.float64)
     n = len(s)
@@ -166,7 +173,7 @@ def alpha_select(s, sig, k: int, lam: float, force_greedy: bool = False) -> Sele
     if n < k:
         k = n
         status = STATUS_SHORT
-    if lam == 0 and not force_greedy:                     # Alg. 1: "top-k fast path"
+    if lam == 0 and not force_greedy:                     # no penalty: plain top-k of the scores
         full = topk_indices(s, n)                         # all indices, best first
         order = full[:k]
         gains = s[order]
@@ -178,57 +185,44 @@ def alpha_select(s, sig, k: int, lam: float, force_greedy: bool = False) -> Sele
                 margins[t] = 0.0
         return Selection(order, gains, margins, np.sort(order), status)
 
-    m = np.zeros(n)                                       # m <- 0_n, S <- {}
-    in_S = np.zeros(n, dtype=bool)
+    red = np.zeros(n)                                     # Eq. 2's max(0, max_j cos) for S = {}
+    chosen = np.zeros(n, dtype=bool)
     order, gains, margins = [], [], []
-
-    def pick(a):
-        i = _argmax_lowest(a, in_S)
-        rest = np.delete(a, i)
-        second = rest.max() if len(rest) else NEG_INF
-        margins.append(a[i] - second if np.isfinite(a[i]) and np.isfinite(second) else
-                       (np.inf if np.isfinite(a[i]) else 0.0))
+    for _t in range(k):
+        gain = s - lam * red                              # Eq. 2 for every candidate
+        gain[chosen] = NEG_INF                            # members of S do not compete
+        i = _argmax_lowest(gain, chosen)                  # Eq. 3
+        others = np.delete(gain, i)
+        second = others.max() if len(others) else NEG_INF
+        margins.append(gain[i] - second if np.isfinite(gain[i]) and np.isfinite(second) else
+                       (np.inf if np.isfinite(gain[i]) else 0.0))
         order.append(i)
-        gains.append(a[i])
-        in_S[i] = True
-        return i
-
-    if k >= 1:
-        a = s.copy()
-        i = pick(a)                                       # i_1 = argmax_i s_i
-        np.maximum(m, sig @ sig[i], out=m)                # m <- max(m, Sims[i_1, :])
-    for _t in range(1, k):                                # t = 1 .. k-1
-        a = s - lam * m                                   # a <- s - lambda m
-        a[in_S] = NEG_INF                                 # a[S] <- -inf
-        i = pick(a)                                       # i <- argmax_j a_j ; S <- S + {i}
-        np.maximum(m, sig @ sig[i], out=m)                # m <- max(m, Sims[i, :])
+        gains.append(gain[i])
+        chosen[i] = True
+        np.maximum(red, sig @ sig[i], out=red)            # cosines of the new member against everyone
     order = np.array(order, dtype=np.int64)
-    return Selection(order, np.array(gains), np.array(margins), np.sort(order), status)  # sort(S)
+    return Selection(order, np.array(gains), np.array(margins), np.sort(order), status)
 
 
-def alpha_select_gram(s, sig, k: int, lam: float) -> np.ndarray:
-    """Algorithm 1 transcribed with the full n x n cosine matrix (tiny n only).
-    Returns sort(S)."""
+def alpha_select_from_definition(s, sig, k: int, lam: float) -> np.ndarray:
+    """The same selection with nothing carried from pick to pick (tiny n only): the cosine
+    matrix of all pairs is formed once, and every pick evaluates Eq. 2 for every candidate
+    from its definition -- the largest cosine against the members chosen so far, floored at
+    zero -- before Eq. 3 takes the best one. Returns the chosen set in ascending order."""
     s, _ = sanitize_scores(s)
     sig = np.asarray(sig, dtype=np.float64)
     n = len(s)
     k = min(k, n)
     if lam == 0:
         return np.sort(topk_indices(s, k))
-    Sims = sig @ sig.T
-    S = []
-    m = np.zeros(n)
-    i1 = _argmax_lowest(s)
-    S.append(i1)
-    m = np.maximum(m, Sims[i1, :])
-    for _t in range(1, k):
-        a = s - lam * m
-        a[S] = NEG_INF
-        taken = np.zeros(n, dtype=bool)
-        taken[S] = True
-        i = _argmax_lowest(a, taken)
-        S.append(i)
-        m = np.maximum(m, Sims[i, :])
+    cosines = sig @ sig.T
+    S: list = []
+    for _t in range(k):
+        gain = np.array([s[i] - (lam * max(0.0, max(cosines[i, j] for j in S)) if S else 0.0) for i in range(n)])
+        member = np.zeros(n, dtype=bool)
+        member[S] = True
+        gain[member] = NEG_INF
+        S.append(_argmax_lowest(gain, member))
     return np.sort(np.array(S, dtype=np.int64))
 
 

@@ -110,7 +110,7 @@ __device__ void greedy_cta(int n, int picks, float lam, bool similarity, int d, 
     const int RPW = 32 / G;                                         // rows per warp and pass
     const int grp = lane / G, lig = lane % G;
     for (int t = 0; t < picks; ++t) {
-        // a = s - lambda m; a[S] = -inf; i = argmax a
+        // Eq. 2 for every candidate still outside the set, Eq. 3's arg-max (ties to the lower slot)
         unsigned long long best = 0ull;
         for (int j = tid; j < n; j += kThreads) {
             if (!taken[j]) {
@@ -132,7 +132,7 @@ __device__ void greedy_cta(int n, int picks, float lam, bool similarity, int d, 
             gain[t] = key_value(best);
             taken[i] = 1;
         }
-        // m <- max(m, Sims[i, :]) with Sims[i, j] = <V_i, V_j> r_i r_j
+        // fold the new member's cosines <V_i, V_j> r_i r_j into every candidate's running maximum
         if (similarity && t + 1 < picks) {
             float vi[8];
             const bool act = lig * 8 < d;

@@ -1,4 +1,4 @@
-"""Helpers for the GPU-vs-oracle parity tests (acceptance rules of the benchmark spec):
+"""Helpers for the GPU-vs-oracle parity tests. Acceptance rules:
 scores within 1e-5 relative (to the Cauchy-Schwarz scale), pick sequences identical
 except where the oracle's own margin is below 1e-6 (checked by replaying the GPU's
 sequence in float64), compacted K/V/pos bit-exact."""

@@ -71,7 +71,7 @@ def test_lambda0_is_topk_in_every_path(seed):
     loop = O.alpha_select(s, sig, k, 0.0, force_greedy=True)
     assert list(fast.order) == want and list(loop.order) == want
     assert list(O.topk_indices(s, k)) == want
-    assert list(O.alpha_select_gram(s, sig, k, 0.0)) == sorted(want)
+    assert list(O.alpha_select_from_definition(s, sig, k, 0.0)) == sorted(want)
     for fg in (False, True):
         oc, _, _, _ = CO.select(s, sig, k, 0.0, force_greedy=fg)
         assert list(oc) == want
@@ -131,7 +131,7 @@ def test_on_demand_rows_equal_full_gram_variant_and_c_twin():
         sig = O.signatures_per_head(V)
         for lam in (0.3, 0.5, 1.0, 2.0):
             a = O.alpha_select(s, sig, k, lam)
-            assert np.array_equal(a.idx_sorted, O.alpha_select_gram(s, sig, k, lam))
+            assert np.array_equal(a.idx_sorted, O.alpha_select_from_definition(s, sig, k, lam))
             oc, gc, mc, st = CO.select(s, sig, k, lam)
             assert np.array_equal(oc, a.order) and st == 0
             assert np.max(np.abs(gc - a.gains)) < 1e-13

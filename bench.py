@@ -2,11 +2,14 @@
 """Benchmark of the KV-cache compression event (fused alpha_compress_event).
 
 One *step* = one pass of the whole hot path (score -> greedy selection -> ordering -> in-place
-compaction) over one batch of synthetic input shaped like the Llama-8B configuration
-(batch 16 x 32 layers x 8 KV heads = 4096 events, N = 192 -> b = 64, d = 128, bf16,
-lambda = 0.5, 5 % near-duplicate V rows). Prints one JSON line.
+compaction) over one batch of synthetic input. The default workload, and the one the headline
+metric is quoted on, is C3: Llama-8B-shaped, batch 16 x 32 layers x 8 KV heads = 4096 events,
+N = 192 -> b = 64, d = 128, bf16, lambda = 0.5, 5 % near-duplicate V rows. `--config` times the
+other four configurations the same way (C4: one step = the batch at lambda 0, 0.5 and 1.0;
+C5: one step = the 32 events of the decode cadence, the refill between them outside the timed
+regions). Prints one JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--config C3] [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
 N > 1 is launched by torch.distributed.run: events are independent, so every rank processes
 its own batch (weak scaling, no data-path collective); the time is the max over ranks.
@@ -29,15 +32,42 @@ if ROOT not in sys.path:
 
 METRIC = "compression events/sec (all layers x KV heads)"
 UNIT = "events/s"
-WORKLOAD = "C3 Llama-8B-shaped: batch 16 x 32 layers x 8 KV heads, N=192 -> b=64, d=128, bf16, lambda=0.5"
-# Algorithmic HBM bytes of one event: read K and V once, write b rows of each, plus positions in,
-# positions + indices out and the query statistic.
+L2_BYTES = 126 * 1024 * 1024
+
+WORKLOADS = {
+    "C1": "C1 single (layer, KV head): N=192 -> b=64, d=128, fp32, lambda=0.5",
+    "C2": "C2 Qwen-7B-shaped: batch 1 x 28 layers x 4 KV heads, N=256 -> b=128, d=128, bf16, lambda=0.5",
+    "C3": "C3 Llama-8B-shaped: batch 16 x 32 layers x 8 KV heads, N=192 -> b=64, d=128, bf16, lambda=0.5",
+    "C4": "C4 large pool: batch 8 x 28 layers x 4 KV heads, N=4096 -> b=128, d=128, bf16, lambda in {0, 0.5, 1.0}",
+    "C5": "C5 decode cadence: batch 64 x 32 layers x 8 KV heads, 32 events of N=256 -> b=128 in a paged buffer, "
+          "d=128, bf16, lambda=0.5",
+}
+# kernel(s) one call of the fused entry point launches for each workload
+KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_tc_kernel<fused>", "C3": "event_tri_kernel<fused>",
+           "C4": "score_kernel + select_pool_kernel + compact_kernel", "C5": "event_tc_kernel<fused>"}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per step from the ncu captures summarised under profiles/,
+# keyed by workload, each with the source revision of csrc/ it was taken at (see kernel_revision()); a
+# capture of another revision is reported as null.
+NCU_TRAFFIC = {
+}
+
+
 def algorithmic_bytes(N, b, d, esize):
+    """HBM bytes one event has to move: read K and V once, write b rows of each, positions in, positions and
+    indices out, the query statistic."""
     return 2 * N * d * esize + 2 * b * d * esize + 4 * N + 8 * b + 4 * d
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on this workload, from
-# the ncu capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 328119296 + 97766400
+
+def kernel_revision():
+    """Hash of the CUDA sources: ties a stored ncu traffic figure to the kernels it was measured on."""
+    import glob
+    import hashlib
+    h = hashlib.sha1()
+    for p in sorted(glob.glob(os.path.join(ROOT, "paper_2605_14292_b200", "csrc", "*"))):
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
 
 
 def load_peaks():
@@ -120,41 +150,74 @@ def events_per_second(events_per_rank: int, world: int, steps: int, total_ms: fl
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle legs
-def oracle_time(ev, reps=1, threads=None):
+def oracle_sample(config: str, seed: int = 0):
+    """A bounded sample of the workload for the CPU oracle: (batch, lambdas, description). The oracle runs
+    whole events of the same seeded recipe; C4 and C5 take a subset of the sequences (C5: its first event)."""
+    from paper_2605_14292_b200 import synth
+    if config == "C1":
+        return synth.make_c1(seed), [0.5], "the single event, 20 repetitions", 20
+    if config == "C2":
+        return synth.make_c2(seed), [0.5], "all 112 events once", 1
+    if config == "C3":
+        return synth.make_c3(seed, B=2), [0.5], "512 of 4096 events (batch 2 of 16)", 1
+    if config == "C4":
+        return synth.make_c4(seed, B=1, L=4, H=4), [0.0, 0.5, 1.0], "16 of 896 events (4 layers of one sequence) at each of the three lambdas", 1
+    c5 = synth.make_c5(seed, B=2, rounds=1)
+    K = synth.paged_gather_dense(c5.pool_K, c5.block_table)
+    V = synth.paged_gather_dense(c5.pool_V, c5.block_table)
+    ev = synth.EventBatch("C5-round0", synth.BF16, K, V, c5.pos, c5.qstat, np.full((2,), 256, dtype=np.int32), c5.budget, c5.lam)
+    return ev, [0.5], "512 of 16384 events (batch 2 of 64), the first of the 32 events only", 1
+
+
+def oracle_time(ev, lams, reps=1, threads=None):
     """Times the C oracle, as it stands, on whole events of `ev` with `threads` host threads."""
     from oracle import c_oracle as CO
     threads = threads or (os.cpu_count() or 1)
     CO.build()
     E = ev.n_events
-    CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, ev.lam, events=(0, min(E, threads)), threads=threads)
+    CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lams[0], events=(0, min(E, threads)), threads=threads)
     t0 = time.perf_counter()
     for _ in range(reps):
-        CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, ev.lam, threads=threads)
+        for lam in lams:
+            CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lam, threads=threads)
     dt = time.perf_counter() - t0
-    return E * reps / dt, threads, dt
+    return E * reps * len(lams) / dt, threads, dt
+
+
+def cpu_baseline(config: str):
+    ev, lams, what, reps = oracle_sample(config)
+    v, threads, dt = oracle_time(ev, lams, reps)
+    # one thread on a smaller slice of the same sample
+    one = ev
+    if ev.n_events > 32:
+        from paper_2605_14292_b200 import synth
+        one = synth.EventBatch(ev.name, ev.dtype, ev.K[:1, :2], ev.V[:1, :2], ev.pos[:1, :2], ev.qstat[:2], ev.p_ref[:1],
+                               ev.budget, ev.lam)
+    v1, _, dt1 = oracle_time(one, lams, reps, threads=1)
+    return {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{what}, C oracle in float64, {dt:.1f} s wall on {threads} threads",
+            "single_thread": {"value": v1, "events": one.n_events * len(lams) * reps, "wall_s": round(dt1, 2)}}
 
 
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    from paper_2605_14292_b200 import synth
-    B_sample = 2                                                     # 512 of the 4096 events per step
-    ev = synth.make_c3(seed=0, B=B_sample)
+    ev, lams, what, reps = oracle_sample(args.config)
     threads = os.cpu_count() or 1
     for _ in range(args.warmup):
-        oracle_time(ev, 1, threads)
+        oracle_time(ev, lams, reps, threads)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_time(ev, 1, threads)
+        oracle_time(ev, lams, reps, threads)
     dt = time.perf_counter() - t0
-    value = ev.n_events * args.steps / dt
-    sample = f"{ev.n_events} of 4096 events per step (batch {B_sample} of 16), C oracle in float64, {threads} threads"
+    value = ev.n_events * len(lams) * reps * args.steps / dt
+    sample = f"per step: {what}, C oracle in float64, {threads} threads"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
+        "config": {"workload": WORKLOADS[args.config], "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -162,7 +225,200 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-# ------------------------------------------------------------------------------------------------ GPU arm
+# ------------------------------------------------------------------------------------------------ GPU workloads
+class DenseWorkload:
+    """C1-C4: a dense batch [B, L, H, N, d]; one step = one fused call per lambda, each on a pristine copy of
+    the batch (the event rewrites its inputs). Pristine copies are restored outside the timed regions."""
+
+    def __init__(self, config, rank, dev, steps, akv, synth, torch):
+        self.akv, self.torch = akv, torch
+        make = {"C1": synth.make_c1, "C2": synth.make_c2, "C3": synth.make_c3, "C4": synth.make_c4}[config]
+        ev = make(seed=rank)
+        self.ev = ev
+        self.lams = [0.0, 0.5, 1.0] if config == "C4" else [ev.lam]
+        B, L, H, N, d = ev.shape
+        self.esize = 2 if ev.dtype == synth.BF16 else 4
+        self.events_per_step = ev.n_events * len(self.lams)
+        self.bytes_per_step = algorithmic_bytes(N, ev.budget, d, self.esize) * self.events_per_step
+        self.launches_hint = len(self.lams)
+        self.LH = L * H
+        self.K0, self.V0, self.P0 = akv.to_device(ev.K, dev), akv.to_device(ev.V, dev), akv.to_device(ev.pos, dev)
+        self.q, self.pref = akv.to_device(ev.qstat, dev), akv.to_device(ev.p_ref, dev)
+        set_bytes = (self.K0.numel() + self.V0.numel()) * self.esize
+        self.set_bytes = set_bytes
+        # how many steps run back to back inside one timed region: bounded by 24 steps and ~40 GB of copies
+        per_step = set_bytes * len(self.lams)
+        self.group = max(1, min(steps, 24, int(40e9 // max(per_step, 1))))
+        self.bufs = [(torch.empty_like(self.K0), torch.empty_like(self.V0), torch.empty_like(self.P0))
+                     for _ in range(self.group * len(self.lams))]
+        self.sel = akv.api._alloc_sel(akv.Layout.dense(self.K0), ev.budget, dev, detail=False)
+        self.opts = [akv.Options(lam=lam) for lam in self.lams]
+        self.flush = None
+        if per_step * self.group < 2 * L2_BYTES:       # working set may stay in L2: evict it before each region
+            self.flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        self.l2 = (f"inputs larger than L2 ({set_bytes / 1e6:.0f} MB per call, fresh copy per call)" if self.flush is None
+                   else f"L2 flushed (a {2 * L2_BYTES >> 20} MiB buffer written) before every timed region; "
+                        f"{set_bytes / 1e6:.2f} MB per call, fresh copy per call")
+
+    def prepare(self, k):
+        for i in range(k * len(self.lams)):
+            self.bufs[i][0].copy_(self.K0); self.bufs[i][1].copy_(self.V0); self.bufs[i][2].copy_(self.P0)
+        if self.flush is not None:
+            self.flush.fill_(1)
+
+    def step(self, i):
+        for j, o in enumerate(self.opts):
+            Kb, Vb, Pb = self.bufs[i * len(self.lams) + j]
+            self.akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, out=self.sel)
+
+    def timed(self, steps, barrier, stream):
+        """Runs `steps` steps in groups; returns the summed device time in ms."""
+        torch = self.torch
+        total, done = 0.0, 0
+        while done < steps:
+            k = min(self.group, steps - done)
+            self.prepare(k)
+            barrier()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            for i in range(k):
+                self.step(i)
+            t1.record(stream)
+            barrier()
+            total += t0.elapsed_time(t1)
+            done += k
+        return total
+
+    def e2e(self, steps, barrier, stream):
+        """Pinned host inputs -> device, the same calls, sorted indices and kept counts back to pinned host
+        memory, all inside the timed region. The compacted K/V rows stay on the device: the cache lives there."""
+        torch, akv = self.torch, self.akv
+        hK, hV, hP = (torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (self.K0, self.V0, self.P0))
+        hK.copy_(self.K0); hV.copy_(self.V0); hP.copy_(self.P0)
+        sel2 = akv.api._alloc_sel(akv.Layout.dense(self.K0), self.ev.budget, self.K0.device, detail=True)
+        h_idx = torch.empty(sel2.idx_sorted.shape, dtype=torch.int32).pin_memory()
+        h_kept = torch.empty(sel2.n_kept.shape, dtype=torch.int32).pin_memory()
+        Kb, Vb, Pb = self.bufs[0]
+
+        def one():
+            for o in self.opts:
+                Kb.copy_(hK, non_blocking=True); Vb.copy_(hV, non_blocking=True); Pb.copy_(hP, non_blocking=True)
+                akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, out=sel2)
+                h_idx.copy_(sel2.idx_sorted, non_blocking=True); h_kept.copy_(sel2.n_kept, non_blocking=True)
+
+        one()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(steps):
+            one()
+        t1.record(stream)
+        barrier()
+        assert int(h_kept.min()) == self.ev.budget
+        h2d = sum(x.numel() * x.element_size() for x in (hK, hV, hP)) * len(self.opts)
+        d2h = sum(x.numel() * x.element_size() for x in (h_idx, h_kept)) * len(self.opts)
+        return t0.elapsed_time(t1), h2d, d2h
+
+
+class CadenceWorkload:
+    """C5: a paged pool; one step = 32 rounds of (compress 256 -> 128 in place, then 128 fresh rows per head
+    appended). Each round's call is timed by its own pair of events; the refill runs between them, untimed."""
+
+    def __init__(self, rank, dev, akv, synth, torch):
+        self.akv, self.torch = akv, torch
+        c5 = synth.make_c5(seed=rank)
+        self.c5 = c5
+        self.rounds = c5.rounds
+        B, L, H, N, d, b = c5.B, c5.L, c5.H, c5.N, c5.d, c5.budget
+        self.esize = 2
+        self.events_per_step = B * L * H * c5.rounds
+        self.bytes_per_step = algorithmic_bytes(N, b, d, 2) * self.events_per_step
+        self.launches_hint = c5.rounds
+        self.LH = L * H
+        self.pool_K0, self.pool_V0 = akv.to_device(c5.pool_K, dev), akv.to_device(c5.pool_V, dev)
+        self.pool_K, self.pool_V = torch.empty_like(self.pool_K0), torch.empty_like(self.pool_V0)
+        self.table = akv.to_device(c5.block_table, dev)
+        self.pos0 = akv.to_device(c5.pos, dev)
+        self.pos = torch.empty_like(self.pos0)
+        self.q = akv.to_device(c5.qstat, dev)
+        self.rK, self.rV = akv.to_device(c5.refill_K, dev), akv.to_device(c5.refill_V, dev)
+        self.lay = akv.Layout.paged(self.pool_K, self.table)
+        self.opts = akv.Options(lam=c5.lam)
+        self.sel = akv.api._alloc_sel(self.lay, b, dev, detail=True)
+        slots = torch.arange(b, N, device=dev)
+        self.pg = self.table.long()[:, (slots // c5.page)]                       # [B, n_new] page of every refilled slot
+        self.off = (slots % c5.page)[None, :].expand(B, -1)
+        self.n_new = N - b
+        self.new_pos = torch.arange(self.n_new, device=dev, dtype=torch.int32)
+        self.set_bytes = (self.pool_K0.numel() + self.pool_V0.numel()) * 2
+        self.l2 = f"inputs larger than L2 ({self.set_bytes / 1e6:.0f} MB touched per event call)"
+
+    def reset(self):
+        self.pool_K.copy_(self.pool_K0); self.pool_V.copy_(self.pool_V0); self.pos.copy_(self.pos0)
+
+    def refill(self, r, srcK=None, srcV=None):
+        c5 = self.c5
+        blk = r % self.rK.shape[0]
+        sK = self.rK[blk] if srcK is None else srcK
+        sV = self.rV[blk] if srcV is None else srcV
+        for l in range(c5.L):
+            self.pool_K[l, self.pg, :, self.off] = sK[l].permute(1, 0, 2)[None].expand(c5.B, -1, -1, -1)
+            self.pool_V[l, self.pg, :, self.off] = sV[l].permute(1, 0, 2)[None].expand(c5.B, -1, -1, -1)
+        self.pos[..., c5.budget:] = c5.N + r * self.n_new + self.new_pos
+
+    def call(self):
+        self.akv.alpha_compress_event(self.pool_K, self.pool_V, self.pos, self.q, self.c5.budget, self.opts,
+                                      layout=self.lay, out=self.sel)
+
+    def timed(self, steps, barrier, stream):
+        torch = self.torch
+        total = 0.0
+        for _ in range(steps):
+            self.reset()
+            pairs = []
+            barrier()
+            for r in range(self.rounds):
+                t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                t0.record(stream)
+                self.call()
+                t1.record(stream)
+                pairs.append((t0, t1))
+                self.refill(r)
+            barrier()
+            total += sum(a.elapsed_time(b) for a, b in pairs)
+        return total
+
+    def e2e(self, steps, barrier, stream):
+        """Per round: the 128 new rows per head come from pinned host memory (copied in and scattered into the
+        pages), then the call, then sorted indices and kept counts back to pinned host memory."""
+        torch = self.torch
+        hK = torch.empty(self.rK[0].shape, dtype=self.rK.dtype).pin_memory()
+        hV = torch.empty(self.rV[0].shape, dtype=self.rV.dtype).pin_memory()
+        hK.copy_(self.rK[0]); hV.copy_(self.rV[0])
+        dK, dV = torch.empty_like(self.rK[0]), torch.empty_like(self.rV[0])
+        h_idx = torch.empty(self.sel.idx_sorted.shape, dtype=torch.int32).pin_memory()
+        h_kept = torch.empty(self.sel.n_kept.shape, dtype=torch.int32).pin_memory()
+        rounds = min(self.rounds, 4)
+        self.reset()
+        self.call()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(steps):
+            for r in range(rounds):
+                dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
+                self.refill(r, dK, dV)
+                self.call()
+                h_idx.copy_(self.sel.idx_sorted, non_blocking=True); h_kept.copy_(self.sel.n_kept, non_blocking=True)
+        t1.record(stream)
+        barrier()
+        assert int(h_kept.min()) == self.c5.budget
+        scale = self.rounds / rounds                                  # reported per step of 32 rounds
+        h2d = (hK.numel() + hV.numel()) * 2 * self.rounds
+        d2h = (h_idx.numel() + h_kept.numel()) * 4 * self.rounds
+        return t0.elapsed_time(t1) * scale, h2d, d2h
+
+
 def run_gpu(args):
     import torch
     import paper_2605_14292_b200 as akv
@@ -178,27 +434,10 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)
     akv.load_library()
 
-    ev = synth.make_c3(seed=rank)                                    # every rank: its own batch of 4096 events
-    B, L, H, N, d = ev.shape
-    E, b = ev.n_events, ev.budget
-    esize = 2
-    opts = akv.Options(lam=ev.lam)
-    K0, V0, P0 = akv.to_device(ev.K, dev), akv.to_device(ev.V, dev), akv.to_device(ev.pos, dev)
-    q, pref = akv.to_device(ev.qstat, dev), akv.to_device(ev.p_ref, dev)
-
-    # The event rewrites K/V/pos in place, so every timed step gets a pristine copy of the batch:
-    # nbuf working sets (each ~405 MB, larger than the 126 MB L2), restored outside the timed regions.
-    nbuf = max(1, min(args.steps, 24))
-    bufs = [(torch.empty_like(K0), torch.empty_like(V0), torch.empty_like(P0)) for _ in range(nbuf)]
-    sel = akv.api._alloc_sel(akv.Layout.dense(K0), b, dev, detail=False)
-
-    def restore(k):
-        for i in range(k):
-            bufs[i][0].copy_(K0); bufs[i][1].copy_(V0); bufs[i][2].copy_(P0)
-
-    def step(i):
-        Kb, Vb, Pb = bufs[i]
-        akv.alpha_compress_event(Kb, Vb, Pb, q, b, opts, p_ref=pref, out=sel)
+    if args.config == "C5":
+        wl = CadenceWorkload(rank, dev, akv, synth, torch)
+    else:
+        wl = DenseWorkload(args.config, rank, dev, args.steps, akv, synth, torch)
 
     def barrier():
         if world > 1:
@@ -206,89 +445,50 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    done = 0
-    while done < args.warmup:
-        k = min(nbuf, args.warmup - done)
-        restore(k)
-        for i in range(k):
-            step(i)
-        done += k
-    torch.cuda.synchronize()
-
     stream = torch.cuda.current_stream()
-    total_ms, done = 0.0, 0
+    wl.timed(args.warmup, barrier, stream)
     launches0 = akv.launch_count()
     with ClockSampler(local_rank) as clocks:
-        while done < args.steps:
-            k = min(nbuf, args.steps - done)
-            restore(k)
-            barrier()
-            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            t0.record(stream)
-            for i in range(k):
-                step(i)
-            t1.record(stream)
-            barrier()
-            total_ms += t0.elapsed_time(t1)
-            done += k
+        total_ms = wl.timed(args.steps, barrier, stream)
     launches = akv.launch_count() - launches0
     total_ms = reduce_max(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
-    value = events_per_second(E, world, args.steps, total_ms)
+    value = events_per_second(wl.events_per_step, world, args.steps, total_ms)
 
-    # roofline of the dominant (only) kernel: algorithmic bytes per launch / mean launch duration
+    # roofline: algorithmic bytes of a step / device time of a step (the step's kernels run back to back on
+    # one stream; for the one-launch routes this is the mean launch duration of the one kernel)
     peak, peak_kind = load_peaks()
-    bytes_per_launch = algorithmic_bytes(N, b, d, esize) * E
-    kernel_ms = ms_per_step                                          # one launch per step, timed back to back
-    achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
+    achieved = wl.bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    rev = kernel_revision()
+    traffic = NCU_TRAFFIC.get(args.config)
+    traffic_bytes = traffic["bytes"] if traffic and traffic.get("revision") == rev else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
-                "kernel": "event_tri_kernel<fused>", "algorithmic_bytes_per_launch": bytes_per_launch}
+                "traffic": traffic_bytes, "peak_kind": f"of {peak_kind}", "kernel": KERNELS[args.config],
+                "algorithmic_bytes_per_step": wl.bytes_per_step, "launches_per_step": launches / args.steps,
+                "frac_of_nominal_8TBs": achieved / 8000.0, "kernel_revision": rev,
+                # bytes the kernels really moved (ncu) over the same time: what the memory system delivered
+                "dram_gbs_from_traffic": None if traffic_bytes is None else traffic_bytes / (ms_per_step * 1e-3) / 1e9,
+                "dram_frac_from_traffic": None if traffic_bytes is None else traffic_bytes / (ms_per_step * 1e-3) / 1e9 / peak}
 
-    # end to end: pinned host buffers -> device, the same C-ABI call, indices and kept counts back
-    hK, hV, hP = (torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (K0, V0, P0))
-    hK.copy_(K0); hV.copy_(V0); hP.copy_(P0)
-    sel2 = akv.api._alloc_sel(akv.Layout.dense(K0), b, dev, detail=True)
-    h_idx = torch.empty(sel2.idx_sorted.shape, dtype=torch.int32).pin_memory()
-    h_kept = torch.empty(sel2.n_kept.shape, dtype=torch.int32).pin_memory()
-    Kb, Vb, Pb = bufs[0]
-    e2e_steps = max(3, min(args.steps, 10))
-
-    def e2e_step():
-        Kb.copy_(hK, non_blocking=True); Vb.copy_(hV, non_blocking=True); Pb.copy_(hP, non_blocking=True)
-        akv.alpha_compress_event(Kb, Vb, Pb, q, b, opts, p_ref=pref, out=sel2)
-        h_idx.copy_(sel2.idx_sorted, non_blocking=True); h_kept.copy_(sel2.n_kept, non_blocking=True)
-
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    t1.record(stream)
-    barrier()
-    e2e_ms = reduce_max(t0.elapsed_time(t1), world, dev)
-    h2d = sum(x.numel() * x.element_size() for x in (hK, hV, hP))
-    d2h = sum(x.numel() * x.element_size() for x in (h_idx, h_kept))
-    e2e = {"value": events_per_second(E, world, e2e_steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "steps": e2e_steps}
-    assert int(h_kept.min()) == b
+    e2e_steps = max(1, min(args.steps, 10 if args.config in ("C1", "C2", "C3") else 2))
+    e2e_ms, h2d, d2h = wl.e2e(e2e_steps, barrier, stream)
+    e2e_ms = reduce_max(e2e_ms, world, dev)
+    e2e = {"value": events_per_second(wl.events_per_step, world, e2e_steps, e2e_ms), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+           "copied_back": "sorted indices and kept counts (the compacted K/V stay on the device)"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, threads, dt = oracle_time(ev, reps=1)
-        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"all {E} events of the same batch once, C oracle in float64, {dt:.1f} s wall"}
+        cpu = cpu_baseline(args.config)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "events_per_gpu": E, "storage": "bf16", "l2": "inputs larger than L2 "
-                       f"({(K0.numel() + V0.numel()) * esize / 1e6:.0f} MB per step, fresh copy per step)",
-                       "sequence_events_per_s": value / (L * H)},
+            "dtype": "bf16" if wl.esize == 2 else "f32", "data": "synthetic",
+            "config": {"workload": WORKLOADS[args.config], "events_per_gpu_per_step": wl.events_per_step,
+                       "storage": "bf16" if wl.esize == 2 else "fp32", "accumulate": "f32", "l2": wl.l2,
+                       "sequence_events_per_s": value / wl.LH},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": clocks.summary(),
         }
@@ -301,12 +501,19 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", default="C3", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="alphakv", choices=["alphakv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = {"C1": 100, "C2": 100, "C3": 100, "C4": 10, "C5": 3}[args.config]
+    if args.warmup is None:
+        args.warmup = 5 if args.config != "C5" else 3
     args.warmup = max(args.warmup, 3)
+    if args.config == "C5":
+        args.warmup = min(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -18,7 +18,7 @@
  *     the legacy default stream). The return code reports host-side validation
  *     and launch errors only; nothing is launched when it is not AKV_OK.
  *   - No exceptions, aborts or exits. akv_last_error() gives a message for the
- *     last failure on the calling thread.
+ *     last failure.
  *   - Tensors are addressed [B, L, H, N, d]: B sequences, L layers, H KV heads,
  *     N slots per (sequence, layer, head), d head dimension (contiguous).
  *     d must be a multiple of 8 and at most 256; row starts must be 16-byte
@@ -53,11 +53,13 @@ typedef enum {
 
 typedef enum { AKV_F32 = 0, AKV_BF16 = 1 } akv_dtype_t;
 
-/* What V-space the cosine of Eq. 2 is taken in. PER_HEAD: the event's own V rows
- * (Eq. 1 with the layer/head sums reduced to the one head; the variant Section 6
- * names). FLAT: Eq. 1 literally, one signature per (sequence, slot) shared by all
- * heads, produced by alpha_signature_flat. */
-typedef enum { AKV_SIG_PER_HEAD = 0, AKV_SIG_FLAT = 1 } akv_sig_mode_t;
+/* What V-space the cosine of Eq. 2 is taken in (Section 6 names the per-head and the
+ * per-layer variant of Eq. 1). PER_HEAD: the event's own V rows (the sums of Eq. 1
+ * reduced to the one head). FLAT: Eq. 1 literally, one signature per (sequence, slot)
+ * shared by all layers and heads, produced by alpha_signature_flat. PER_LAYER: the
+ * sum of Eq. 1 taken over the KV heads of one layer only, one signature per
+ * (sequence, layer, slot), produced by alpha_signature_layer. */
+typedef enum { AKV_SIG_PER_HEAD = 0, AKV_SIG_FLAT = 1, AKV_SIG_PER_LAYER = 2 } akv_sig_mode_t;
 
 /* Layout of K and of V (both use the same one). Strides are in ELEMENTS.
  * Dense (page_size == 0): row (b,l,h,n) starts at
@@ -79,6 +81,10 @@ typedef struct {
 
 #define AKV_FLAG_FORCE_GREEDY 1u /* run the greedy loop even at lambda == 0 (testing aid) */
 #define AKV_FLAG_NO_PRUNE 2u     /* never shrink the candidate pool before the loop (testing aid) */
+/* Testing aid for the bounded waits of the fused on-chip kernels: no K row is requested and the
+ * waits poll only a few times, so every wait runs out with nothing in flight; each event then
+ * reports status 3 and K, V and pos are left as they were. */
+#define AKV_FLAG_TEST_STARVE_WAIT 4u
 
 typedef struct {
     float lambda;          /* >= 0; 0 takes the top-k branch of Algorithm 1 */
@@ -87,18 +93,37 @@ typedef struct {
     int32_t future_window; /* W >= 1 future query positions averaged by the score; default 1 */
     akv_sig_mode_t sig_mode;
     uint32_t flags;
+    /* Per-(layer, head) budgets (Section 2 "Budget-allocation compression", Section 6: alpha as the
+     * scorer inside a per-head or per-layer budget allocator): device int32 [L, H], or NULL for the
+     * same budget everywhere. Event (b, l, h) keeps min(head_budgets[l*H + h], n_cand) rows; every
+     * entry must lie in 1..budget, where the call's `budget` argument is the largest of them and
+     * stays the row length of idx_sorted / pick_order / pick_gain (unused entries -1 / -1 / 0). */
+    const int32_t* head_budgets;
 } akv_options_t;
 
 /* Fills *opt with the defaults named above (lambda = 0.5, the value the paper settles on). */
 void akv_default_options(akv_options_t* opt);
 
 /* Creates a handle bound to CUDA device `device`. The handle keeps a grow-only
- * scratch buffer (cudaMalloc on first need, freed by akv_destroy). One handle
- * must not be used from two host threads at once. */
+ * scratch buffer (cudaMalloc on first need, freed by akv_destroy; akv_workspace_bytes
+ * tells how large a call needs it). One handle must not be used from two host threads
+ * at once, and every call on one handle shares that scratch: two calls that use it and
+ * whose kernels overlap on the GPU (different streams, no ordering between them) race
+ * on it -- order such calls, or give each stream its own handle. */
 akv_status_t akv_create(akv_handle_t** out, int device);
 akv_status_t akv_destroy(akv_handle_t* h);
-/* Message for the most recent error on the calling thread; static storage. */
-const char* akv_last_error(void);
+/* Message of the most recent failed call on handle `h` (storage inside the handle, valid
+ * until the next failure or akv_destroy). With h == NULL: the most recent failure on the
+ * calling thread, whichever handle it was on -- the only way to read why akv_create
+ * failed or what a call given a NULL handle complained about. */
+const char* akv_last_error(const akv_handle_t* h);
+/* Bytes of handle scratch that alpha_compress_event needs for this layout, budget and
+ * options when its `scores` argument is NULL: 0 when the event runs in one launch with
+ * everything on chip, else the B*L*H*N fp32 scores that pass from the scoring launch to
+ * the selection launch. The answer depends on the current device's shared-memory size.
+ * Callers that cannot tolerate a cudaMalloc inside the call can pass their own `scores`
+ * buffer (then no scratch is used) or use alpha_compress_event_static. */
+akv_status_t akv_workspace_bytes(const akv_layout_t* lay, int32_t budget, const akv_options_t* opt, size_t* bytes);
 const char* akv_status_string(akv_status_t s);
 /* Number of kernels this library has launched so far in this process. */
 uint64_t akv_launch_count(void);
@@ -133,8 +158,11 @@ akv_status_t alpha_score(akv_handle_t* h, const akv_layout_t* lay, const void* K
  * top-k when lambda == 0. fp32 accumulation; cos(v_i, v_j) = <V_i, V_j> r_i r_j
  * with r = 1 / (||V||_2 + eps) (Eq. 1's normalisation).
  *   scores     device fp32 [B, L, H, N] in.
- *   V          device, layout `lay`, read only (PER_HEAD mode); may be NULL in FLAT mode.
- *   flat_sig   device fp32 [B, N, d], FLAT mode only (from alpha_signature_flat), else NULL.
+ *   V          device, layout `lay`, read only (PER_HEAD mode); may be NULL in the other modes.
+ *   flat_sig   device fp32 signatures: [B, N, d] in FLAT mode (from alpha_signature_flat),
+ *              [B, L, N, d] in PER_LAYER mode (from alpha_signature_layer), NULL in PER_HEAD mode.
+ *   Limits: the general selection kernel keeps per-candidate state in shared memory, which bounds
+ *   N at about 10 000 (AKV_ERR_UNSUPPORTED beyond).
  *   budget     1 <= budget <= N (the paper's k).
  *   idx_sorted device int32 [B, L, H, budget] out: sort(S), ascending slot index.
  *   pick_order device int32 [B, L, H, budget] out or NULL: i_1, i_2, ... in pick order.
@@ -154,6 +182,16 @@ akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, const float*
 akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, const void* V,
                                   const int32_t* n_cand, const akv_options_t* opt, float* flat_sig,
                                   void* stream);
+
+/*
+ * alpha_signature_layer -- the per-layer variant of Eq. 1 that Section 6 names: the sum runs over the
+ * KV heads of one layer, u_i^(l) = (1/H) sum_h V_i^(l,h), v_i^(l) = u_i^(l) / (||u_i^(l)||_2 + eps).
+ *   layer_sig  device fp32 [B, L, N, d] out (unit-normalised rows); pass it as `flat_sig` with
+ *              sig_mode = AKV_SIG_PER_LAYER.
+ */
+akv_status_t alpha_signature_layer(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+                                   const int32_t* n_cand, const akv_options_t* opt, float* layer_sig,
+                                   void* stream);
 
 /*
  * kv_compact -- the retained rows become the new cache of at most `budget` rows

@@ -175,12 +175,14 @@ static int cmp_i64(const void* x, const void* y) {
  * events e0 <= e < e1. pos is [E, n] or NULL; qstat [L*H, d]; p_ref [B] or NULL
  * (then max position + 1 of the event). Outputs (any may be NULL): scores [E, n],
  * idx_sorted [E, k] (int32, -1 padded), order [E, k], Kout/Vout [E, k, d] raw
- * copies, posout [E, k]. */
+ * copies, posout [E, k]. budgets: NULL, or [L*H] per-(layer, head) budgets (each <= k, the
+ * row length of the outputs): event (b, l, h) then keeps budgets[l*H + h] rows (Section 6: the
+ * selector used inside a per-head or per-layer budget allocator). */
 void orc_event_batch(const void* K, const void* V, int dtype, int B, int L, int H, int n, int d,
                      const int32_t* pos, const float* qstat, const int32_t* p_ref, int W, double base,
                      double eps, int k, double lam, int force_greedy, int e0, int e1, double* scores,
                      int32_t* idx_sorted, int32_t* order_out, void* Kout, void* Vout, int32_t* posout,
-                     int32_t* status_out) {
+                     int32_t* status_out, const int32_t* budgets) {
     (void)B;
     const size_t es = dtype == ORC_BF16 ? 2 : 4;
     double* s = (double*)malloc(sizeof(double) * n);
@@ -206,7 +208,8 @@ void orc_event_batch(const void* K, const void* V, int dtype, int B, int L, int 
         orc_score(Ke, dtype, n, d, pe, qstat + (size_t)lh * d, pr, W, base, s);
         orc_signature(Ve, dtype, n, d, eps, sig);
         int st = 0;
-        int kk = orc_select(s, sig, n, d, k, lam, force_greedy, order, gain, margin, &st);
+        const int k_event = budgets ? (budgets[lh] < k ? budgets[lh] : k) : k;
+        int kk = orc_select(s, sig, n, d, k_event, lam, force_greedy, order, gain, margin, &st);
         if (scores) memcpy(scores + (size_t)e * n, s, sizeof(double) * n);
         if (order_out)
             for (int t = 0; t < k; ++t) order_out[(size_t)e * k + t] = t < kk ? (int32_t)order[t] : -1;

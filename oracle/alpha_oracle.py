@@ -120,6 +120,17 @@ def signatures_flat(V_all, eps: float = 1e-8) -> np.ndarray:
     return u / (nrm + eps)[:, None]
 
 
+def signatures_per_layer(V_layer, eps: float = 1e-8) -> np.ndarray:
+    """The per-layer variant Section 6 names: Eq. 1 with the sum restricted to the H KV heads
+    of one layer, u_i = (1/H) sum_h V_i^(h);  v_i = u_i / (||u_i||_2 + eps).
+    V_layer is [H, n, d] for one (sequence, layer)."""
+    V_layer = widen(V_layer)
+    H, n, d = V_layer.shape
+    u = V_layer.sum(axis=0) / H
+    nrm = np.sqrt((u * u).sum(axis=1))
+    return u / (nrm + eps)[:, None]
+
+
 # --------------------------------------------------------------------------- selection
 def _argmax_lowest(a: np.ndarray, excluded: Optional[np.ndarray] = None) -> int:
     """argmax over the candidates not in ``excluded``, ties to the lowest index.

@@ -78,10 +78,11 @@ def select(s, sig, k, lam, force_greedy=False):
 
 
 def event_batch(K, V, pos, qstat, p_ref, k, lam, W=1, base=10000.0, eps=1e-8, force_greedy=False,
-                events=None, threads=1, want_rows=True, want_scores=True):
+                events=None, threads=1, want_rows=True, want_scores=True, budgets=None):
     """Run whole events over a dense batch [B, L, H, n, d]; returns a dict of
     arrays shaped [B, L, H, ...]. ``events`` = (e0, e1) range in flattened
-    (b, l, h) order (default all); outside it outputs are left untouched (zeros)."""
+    (b, l, h) order (default all); outside it outputs are left untouched (zeros). ``budgets``: optional int32
+    [L, H] per-(layer, head) budgets (each <= k; k stays the row length of the outputs)."""
     K = np.ascontiguousarray(K)
     V = np.ascontiguousarray(V)
     B, L, H, n, d = K.shape
@@ -91,6 +92,7 @@ def event_batch(K, V, pos, qstat, p_ref, k, lam, W=1, base=10000.0, eps=1e-8, fo
     pp = None if pos is None else np.ascontiguousarray(pos, dtype=np.int32).reshape(E, n)
     q = np.ascontiguousarray(qstat, dtype=np.float32)
     pr = None if p_ref is None else np.ascontiguousarray(p_ref, dtype=np.int32)
+    bud = None if budgets is None else np.ascontiguousarray(budgets, dtype=np.int32).reshape(L * H)
     out = {
         "scores": np.zeros((B, L, H, n), dtype=np.float64) if want_scores else None,
         "idx_sorted": np.full((B, L, H, k), -1, dtype=np.int32),
@@ -106,7 +108,7 @@ def event_batch(K, V, pos, qstat, p_ref, k, lam, W=1, base=10000.0, eps=1e-8, fo
                               C.c_int(d), _p(pp), _p(q), _p(pr), C.c_int(W), C.c_double(base),
                               C.c_double(eps), C.c_int(k), C.c_double(lam), C.c_int(int(force_greedy)),
                               C.c_int(lo), C.c_int(hi), _p(out["scores"]), _p(out["idx_sorted"]),
-                              _p(out["order"]), _p(out["K"]), _p(out["V"]), _p(out["pos"]), _p(out["status"]))
+                              _p(out["order"]), _p(out["K"]), _p(out["V"]), _p(out["pos"]), _p(out["status"]), _p(bud))
 
     threads = max(1, int(threads))
     if threads == 1 or e1 - e0 < 2:

@@ -19,13 +19,14 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_PKG, "libalphakv.so")
 
 AKV_F32, AKV_BF16 = 0, 1
-SIG_PER_HEAD, SIG_FLAT = 0, 1
+SIG_PER_HEAD, SIG_FLAT, SIG_PER_LAYER = 0, 1, 2
 FLAG_FORCE_GREEDY = 1
 FLAG_NO_PRUNE = 2
+FLAG_TEST_STARVE_WAIT = 4
 
 EXPORTS = ("akv_default_options", "akv_create", "akv_destroy", "akv_last_error", "akv_status_string",
-           "akv_launch_count", "alpha_score", "alpha_select", "alpha_signature_flat", "kv_compact",
-           "alpha_compress_event", "alpha_compress_event_static")
+           "akv_launch_count", "akv_workspace_bytes", "alpha_score", "alpha_select", "alpha_signature_flat",
+           "alpha_signature_layer", "kv_compact", "alpha_compress_event", "alpha_compress_event_static")
 
 
 class AkvError(RuntimeError):
@@ -44,7 +45,7 @@ class _Layout(C.Structure):
 
 class _Options(C.Structure):
     _fields_ = [("lam", C.c_float), ("eps", C.c_float), ("rope_base", C.c_float), ("future_window", C.c_int32),
-                ("sig_mode", C.c_int), ("flags", C.c_uint32)]
+                ("sig_mode", C.c_int), ("flags", C.c_uint32), ("head_budgets", C.c_void_p)]
 
 
 _lib = None
@@ -61,6 +62,7 @@ def load_library(path: Optional[str] = None):
                           "(there is no CPU fallback)")
     lib = C.CDLL(p)
     lib.akv_last_error.restype = C.c_char_p
+    lib.akv_last_error.argtypes = [C.c_void_p]
     lib.akv_status_string.restype = C.c_char_p
     lib.akv_launch_count.restype = C.c_uint64
     lib.akv_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
@@ -69,6 +71,8 @@ def load_library(path: Optional[str] = None):
     lib.alpha_score.argtypes = [vp, C.POINTER(_Layout), vp, vp, i64, i64, i64, vp, vp, vp, C.POINTER(_Options), vp, vp, vp]
     lib.alpha_select.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, vp, i32, C.POINTER(_Options), vp, vp, vp, vp, vp, vp]
     lib.alpha_signature_flat.argtypes = [vp, C.POINTER(_Layout), vp, vp, C.POINTER(_Options), vp, vp]
+    lib.alpha_signature_layer.argtypes = [vp, C.POINTER(_Layout), vp, vp, C.POINTER(_Options), vp, vp]
+    lib.akv_workspace_bytes.argtypes = [C.POINTER(_Layout), i32, C.POINTER(_Options), C.POINTER(C.c_size_t)]
     lib.kv_compact.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, i32, vp]
     lib.alpha_compress_event.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32,
                                          C.POINTER(_Options), vp, vp, vp, vp, vp, vp, vp]
@@ -93,7 +97,7 @@ def _handle(device: torch.device):
 
 def _check(code: int):
     if code != 0:
-        raise AkvError(code, load_library().akv_last_error().decode())
+        raise AkvError(code, load_library().akv_last_error(None).decode())
 
 
 def launch_count() -> int:
@@ -108,9 +112,14 @@ class Options:
     future_window: int = 1
     sig_mode: int = SIG_PER_HEAD
     flags: int = 0
+    head_budgets: Optional[torch.Tensor] = None   # device int32 [L, H]: per-(layer, head) budgets, or None
 
     def c(self) -> _Options:
-        return _Options(self.lam, self.eps, self.rope_base, self.future_window, self.sig_mode, self.flags)
+        hb = self.head_budgets
+        if hb is not None and (hb.dtype != torch.int32 or not hb.is_cuda or not hb.is_contiguous()):
+            raise ValueError("head_budgets must be a contiguous int32 CUDA tensor [L, H]")
+        return _Options(self.lam, self.eps, self.rope_base, self.future_window, self.sig_mode, self.flags,
+                        None if hb is None else hb.data_ptr())
 
 
 @dataclass
@@ -279,6 +288,27 @@ def alpha_signature_flat(V, opts: Optional[Options] = None, n_cand=None, layout:
         _check(load_library().alpha_signature_flat(_handle(V.device), C.byref(lay.c()), _ptr(V), _ptr(n_cand),
                                                    C.byref(opts.c()), _ptr(out), _stream()))
     return out
+
+
+def alpha_signature_layer(V, opts: Optional[Options] = None, n_cand=None, layout: Optional[Layout] = None, out=None):
+    """Per-layer signatures [B, L, N, d] (fp32), Eq. 1 summed over one layer's heads -- C entry point
+    ``alpha_signature_layer``."""
+    lay = _lay(V, layout)
+    opts = opts or Options()
+    if out is None:
+        out = torch.zeros((lay.B, lay.L, lay.N, lay.d), dtype=torch.float32, device=V.device)
+    _need(out, torch.float32, "out")
+    with torch.cuda.device(V.device):
+        _check(load_library().alpha_signature_layer(_handle(V.device), C.byref(lay.c()), _ptr(V), _ptr(n_cand),
+                                                    C.byref(opts.c()), _ptr(out), _stream()))
+    return out
+
+
+def workspace_bytes(layout: Layout, budget: int, opts: Optional[Options] = None) -> int:
+    """Scratch bytes the fused call would allocate for this shape -- C entry point ``akv_workspace_bytes``."""
+    out = C.c_size_t(0)
+    _check(load_library().akv_workspace_bytes(C.byref(layout.c()), budget, C.byref((opts or Options()).c()), C.byref(out)))
+    return int(out.value)
 
 
 def kv_compact(K, V, pos, idx_sorted, layout: Optional[Layout] = None):

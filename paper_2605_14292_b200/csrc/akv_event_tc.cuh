@@ -73,9 +73,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after a fixed number of polls instead of spinning for ever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (int it = 0; it < kWaitPolls; ++it)
+// Bounded wait: gives up after `polls` polls instead of spinning for ever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int polls) {
+    for (int it = 0; it < polls; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     const EventId id = decode_event(lay, blockIdx.x);
     const int n = event_n(a, id.b);
     const int N = lay.N;
-    const int picks = min(a.budget, n);
+    const int bud = event_budget(a, id);
+    const int picks = min(bud, n);
     const TcSmem sp = plan_tc_smem(N, a.budget);
     unsigned char* tile = smem + sp.tile;
     float* s = reinterpret_cast<float*>(smem + sp.s);
@@ -241,7 +242,9 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         // instruction, so a copy per thread costs a dozen issue slots each)
         if (tid == 0) {
             mbar_expect_tx(barK, (uint32_t)n * 256u);
-            if (lay.page_size == 0 && lay.sn == kTcD) {
+            if (a.starve) {
+                // testing aid: nothing is requested, the wait below runs out
+            } else if (lay.page_size == 0 && lay.sn == kTcD) {
                 const __nv_bfloat16* k0 = Kg + rowoff(0);
                 for (int row = 0; row < n; row += 128)  // 32 KB pieces
                     bulk_g2s(tile_u32 + row * 256, k0 + (long long)row * kTcD, (uint32_t)min(128, n - row) * 256u, barK);
@@ -294,7 +297,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         } else {
             __syncthreads();
         }
-        timeout = !mbar_wait_bounded(barK, 0);
+        timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
         if (!timeout) {
             for (int j0 = 4 * warp; j0 < n; j0 += 4 * (kTcThreads / 32)) {
                 const int j = j0 + grp;
@@ -354,7 +357,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     timeout = __syncthreads_or(timeout);
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
-        mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
+        mbar_wait_bounded(barK, 0, a.wait_polls);  // give copies still in flight another bounded chance to land
         return;
     }
     bad = __syncthreads_or(bad);
@@ -475,7 +478,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
             }
         }
     }
-    if (do_mma) timeout = !mbar_wait_bounded(barM, 0);
+    if (do_mma) timeout = !mbar_wait_bounded(barM, 0, a.wait_polls);
     tc_fence_after();
     timeout = __syncthreads_or(timeout);
     if (timeout) {
@@ -606,7 +609,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     }
     if (tid == 0) {
         if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
     }
     if (!FUSED) return;
 

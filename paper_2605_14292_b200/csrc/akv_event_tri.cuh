@@ -231,7 +231,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     const EventId id = decode_event(lay, blockIdx.x);
     const int n = event_n(a, id.b);
     const int N = lay.N;
-    const int picks = min(a.budget, n);
+    const int bud = event_budget(a, id);
+    const int picks = min(bud, n);
     const TriSmem sp = plan_tri_smem(N, a.budget);
     unsigned char* tile = smem + sp.tile;
     float* tri = reinterpret_cast<float*>(tile);  // lower triangle of the cosine matrix, after the product
@@ -276,7 +277,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     // thread (a bulk copy is a per-warp instruction)
     auto request_k_rows = [&](int r0, int r1, int slot0, uint32_t bar) {
         mbar_expect_tx(bar, (uint32_t)(r1 - r0) * 256u);
-        for (int row = r0; row < r1;) {
+        for (int row = r0; row < r1 && !a.starve;) {  // starve (testing aid): nothing is requested, the waits run out
             int run = 1;
             if (dense && lay.sn == kTcD) run = min(r1 - row, 128);
             else if (!dense && lay.s_page_n == kTcD) run = min(r1 - row, lay.page_size - row % lay.page_size);
@@ -393,12 +394,12 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
                 }
             }
         };
-        timeout = !mbar_wait_bounded(barK, 0);
+        timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
         const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
             // first and third stretch share one copy of the loop (the kernel's code should stay small)
-            if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0);
+            if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0, a.wait_polls);
             score_rounds(pass ? kTriTileRows / 16 : 0, pass ? rounds : late_round);
             if (!pass) {
                 if (n_late > 0) {
@@ -423,8 +424,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     timeout = __syncthreads_or(timeout);
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
-        mbar_wait_bounded(barK, 0);  // give copies still in flight another bounded chance to land
-        if (n_late > 0) mbar_wait_bounded(barL, 0);
+        mbar_wait_bounded(barK, 0, a.wait_polls);  // give copies still in flight another bounded chance to land
+        if (n_late > 0) mbar_wait_bounded(barL, 0, a.wait_polls);
         if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
         return;
     }
@@ -506,7 +507,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
             }
             umma_commit(barM);
         }
-        timeout = !mbar_wait_bounded(barM, 0);
+        timeout = !mbar_wait_bounded(barM, 0, a.wait_polls);
         tc_fence_after();
     }
     timeout = __syncthreads_or(timeout);  // also: the product has read the whole tile before the triangle lands on it
@@ -630,7 +631,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     }
     if (tid == 0) {
         if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
     }
     if (!FUSED) return;
 

@@ -12,12 +12,16 @@ struct EventArgs {
     const int* n_cand;      // [B] or null
     const float* qstat;     // [L,H,d]
     const int* p_ref;       // [B] or null
-    const float* flat_sig;  // [B,N,d] or null (flat signature mode)
-    int budget;
+    const float* flat_sig;  // shared signatures, or null: [B,N,d] (Eq. 1) or [B,L,N,d] (per layer)
+    long long sig_sb, sig_sl;  // element strides of flat_sig over sequences and layers (0 for the flat mode's layers)
+    const int* head_budgets;   // [L,H] or null: per-(layer, head) budgets, each <= budget
+    int budget;             // largest budget of the call = row length of the index outputs
     float lam, eps;
     int greedy;             // 1: run the loop with similarity updates; 0: top-k
     int no_prune;           // 1: keep every candidate in the pool the loop runs over
     int tmem_cols;          // tensor-memory columns the tensor-memory kernel claims per CTA (0: none)
+    int starve;             // testing aid: request no K row, so that the bounded waits run out
+    int wait_polls;         // polls after which a bounded wait gives up
     int* idx_sorted;
     int* pick_order;
     float* pick_gain;
@@ -29,6 +33,17 @@ struct EventArgs {
 __device__ __forceinline__ int event_n(const EventArgs& a, int b) {
     int n = a.n_cand ? a.n_cand[b] : a.lay.N;
     return n < 0 ? 0 : (n > a.lay.N ? a.lay.N : n);
+}
+
+// rows this event keeps at most: its (layer, head) budget when budgets are given per head
+__device__ __forceinline__ int event_budget(const EventArgs& a, const EventId& id) {
+    if (!a.head_budgets) return a.budget;
+    const int b = a.head_budgets[id.l * a.lay.H + id.h];
+    return b < 1 ? 1 : (b > a.budget ? a.budget : b);
+}
+// shared signature rows of this event's (sequence, layer)
+__device__ __forceinline__ const float* event_sig(const EventArgs& a, const EventId& id) {
+    return a.flat_sig + id.b * a.sig_sb + id.l * a.sig_sl;
 }
 
 __device__ __forceinline__ const int* event_pos(const PosDesc& p, const EventId& id) {
@@ -154,9 +169,10 @@ __global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArg
     bad = __syncthreads_or(bad);
 
     // selection
-    const int picks = min(a.budget, n);
+    const int bud = event_budget(a, id);
+    const int picks = min(bud, n);
     if (a.flat_sig) {
-        StridedRows<float> rows{a.flat_sig + (long long)id.b * N * d, d};
+        StridedRows<float> rows{event_sig(a, id), d};
         greedy_cta<float>(n, picks, a.lam, a.greedy != 0, d, s, nullptr, m, taken, order, gain, rows, red);
     } else {
         StridedRows<T> rows{Vt, d};
@@ -174,7 +190,7 @@ __global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArg
     }
     if (tid == 0) {
         if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
     }
     // compaction: kept rows go to slots 0..picks-1 of the same buffer (all sources are on chip)
     const int cpr = d * (int)sizeof(T) / 16;
@@ -192,7 +208,8 @@ __global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArg
 }
 
 // ---------------------------------------------------------------------------------------------
-// Stand-alone score: grid (row blocks, events); K streamed from global memory once.
+// Stand-alone score: one CTA per (event, block of kScoreRows rows), both folded into grid.x; K
+// streamed from global memory once.
 // ---------------------------------------------------------------------------------------------
 constexpr int kScoreRows = 64;  // rows per CTA
 
@@ -202,10 +219,11 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, cons
     __shared__ float2 g[kMaxHalf];
     __shared__ int redi[kWarps];
     const DevLayout& lay = a.lay;
-    const EventId id = decode_event(lay, blockIdx.y);
+    const int row_blocks = (lay.N + kScoreRows - 1) / kScoreRows;
+    const EventId id = decode_event(lay, blockIdx.x / row_blocks);
     const int n = event_n(a, id.b);
     const int d = lay.d;
-    const int row0 = blockIdx.x * kScoreRows;
+    const int row0 = (blockIdx.x % row_blocks) * kScoreRows;
     if (row0 >= n) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int* gpos = event_pos(a.pos, id);
@@ -313,20 +331,24 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const CompactArgs a) 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Eq. 1: flat signature. One warp group per (sequence, slot): u = mean over (l, h) of V rows,
-// v = u / (||u|| + eps), written as fp32 [B, N, d].
+// Eq. 1: shared signatures. One warp group per (sequence, slot): u = mean over (l, h) of V rows,
+// v = u / (||u|| + eps), written as fp32 [B, N, d]; per_layer: one group per (sequence, layer, slot),
+// the mean runs over the heads of that layer only, written as fp32 [B, L, N, d].
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kThreads) flat_signature_kernel(const DevLayout lay, const void* V, const int* n_cand,
-                                                                 float eps, float* out) {
+                                                                 float eps, float* out, int per_layer) {
     const int d = lay.d;
     const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
     const int RPW = 32 / G;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int grp = lane / G, lig = lane % G;
-    const long long slot = ((long long)blockIdx.x * kWarps + warp) * RPW + grp;  // over B*N
-    const bool inrange = slot < (long long)lay.B * lay.N;
-    const int b = inrange ? (int)(slot / lay.N) : 0;
+    const int groups = per_layer ? lay.B * lay.L : lay.B;
+    const long long slot = ((long long)blockIdx.x * kWarps + warp) * RPW + grp;  // over groups * N
+    const bool inrange = slot < (long long)groups * lay.N;
+    const int grpi = inrange ? (int)(slot / lay.N) : 0;
+    const int b = per_layer ? grpi / lay.L : grpi;
+    const int l0 = per_layer ? grpi % lay.L : 0, l1 = per_layer ? l0 + 1 : lay.L;
     const int j = inrange ? (int)(slot % lay.N) : 0;
     int n = n_cand ? n_cand[b] : lay.N;
     n = n < 0 ? 0 : (n > lay.N ? lay.N : n);
@@ -335,14 +357,14 @@ __global__ void __launch_bounds__(kThreads) flat_signature_kernel(const DevLayou
     const T* Vg = reinterpret_cast<const T*>(V);
     float u[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (act) {
-        for (int l = 0; l < lay.L; ++l)
+        for (int l = l0; l < l1; ++l)
             for (int h = 0; h < lay.H; ++h) {
                 float x[8];
                 load8(Vg + row_offset(lay, b, l, h, j) + lig * 8, x);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) u[q] += x[q];
             }
-        const float inv = 1.f / (float)(lay.L * lay.H);
+        const float inv = 1.f / (float)((l1 - l0) * lay.H);
 #pragma unroll
         for (int q = 0; q < 8; ++q) u[q] *= inv;
     }

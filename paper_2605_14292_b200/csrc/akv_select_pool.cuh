@@ -85,7 +85,8 @@ __global__ void __launch_bounds__(kThreads) select_pool_kernel(const EventArgs a
     T* tile = reinterpret_cast<T*>(smem + sp.tile);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool similarity = a.greedy != 0;
-    const int picks = min(a.budget, n);
+    const int bud = event_budget(a, id);
+    const int picks = min(bud, n);
 
     int bad = 0;
     for (int j = tid; j < n; j += kThreads) {
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(kThreads) select_pool_kernel(const EventArgs a
     }
 
     // ---- the pool's rows: into the tile when they fit, reciprocal norms (Eq. 1) ---------------------------
-    const T* gbase = FLAT ? reinterpret_cast<const T*>(a.flat_sig) + (long long)id.b * N * d : reinterpret_cast<const T*>(a.V);
+    const T* gbase = FLAT ? reinterpret_cast<const T*>(event_sig(a, id)) : reinterpret_cast<const T*>(a.V);
     PoolLayoutRows<T> lrows{gbase, &lay, id.b, id.l, id.h, pool};
     PoolStridedRows<T> frows{gbase, d, pool};
     StridedRows<T> trows{tile, d};
@@ -187,7 +188,7 @@ __global__ void __launch_bounds__(kThreads) select_pool_kernel(const EventArgs a
     }
     if (tid == 0) {
         if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < a.budget ? 2 : (bad ? 1 : 0);
+        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
     }
 }
 

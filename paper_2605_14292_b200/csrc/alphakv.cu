@@ -23,6 +23,7 @@ struct akv_handle {
     ScoreTab tab;
     float tab_base;
     int tab_d, tab_W;
+    char err[512];     // message of the last failed call on this handle
 };
 
 static thread_local char g_err[512] = "";
@@ -41,7 +42,16 @@ static akv_status_t fail(akv_status_t s, const char* fmt, ...) {
         if (e_ != cudaSuccess) return fail(AKV_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
     } while (0)
 
-extern "C" const char* akv_last_error(void) { return g_err; }
+// Failures are formatted into a thread-local buffer (a failure can precede any handle: akv_create
+// itself, a NULL handle); calls that have a handle also leave the message there.
+extern "C" const char* akv_last_error(const akv_handle_t* h) { return h ? h->err : g_err; }
+static akv_status_t finish(akv_handle* h, akv_status_t s) {
+    if (h && s != AKV_OK) {
+        strncpy(h->err, g_err, sizeof(h->err) - 1);
+        h->err[sizeof(h->err) - 1] = 0;
+    }
+    return s;
+}
 extern "C" uint64_t akv_launch_count(void) { return g_launches.load(); }
 extern "C" const char* akv_status_string(akv_status_t s) {
     switch (s) {
@@ -170,7 +180,8 @@ static akv_status_t check_options(const akv_options_t* o) {
     if (!(o->eps >= 0.f) || !std::isfinite(o->eps)) return fail(AKV_ERR_INVALID_ARG, "eps must be finite and >= 0");
     if (!(o->rope_base > 0.f) || !std::isfinite(o->rope_base)) return fail(AKV_ERR_INVALID_ARG, "rope_base must be positive");
     if (o->future_window < 1 || o->future_window > 65536) return fail(AKV_ERR_INVALID_ARG, "future_window must be in 1..65536");
-    if (o->sig_mode != AKV_SIG_PER_HEAD && o->sig_mode != AKV_SIG_FLAT) return fail(AKV_ERR_UNSUPPORTED, "sig_mode %d", (int)o->sig_mode);
+    if (o->sig_mode != AKV_SIG_PER_HEAD && o->sig_mode != AKV_SIG_FLAT && o->sig_mode != AKV_SIG_PER_LAYER)
+        return fail(AKV_ERR_UNSUPPORTED, "sig_mode %d", (int)o->sig_mode);
     return AKV_OK;
 }
 
@@ -235,14 +246,20 @@ struct DeviceGuard {
 // ------------------------------------------------------------------------------------------------
 // launch helpers
 // ------------------------------------------------------------------------------------------------
-static akv_status_t launch_score(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+// Every launch helper takes `dry`: with it set, the helper performs its checks and one-time kernel
+// attribute calls and returns before launching, so that a call made of several launches can be
+// refused as a whole before its first kernel is enqueued.
+static akv_status_t launch_score(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
+    const long long blocks = (long long)((a.lay.N + kScoreRows - 1) / kScoreRows) * E;
+    if (blocks > INT_MAX) return fail(AKV_ERR_UNSUPPORTED, "alpha_score: %lld row blocks exceed the grid limit", blocks);
+    if (dry) return AKV_OK;
     if (a.status) {
         fill_int_kernel<<<(E + 255) / 256, 256, 0, st>>>(a.status, E, 0);
         akv_status_t s = launched("fill");
         if (s != AKV_OK) return s;
     }
-    dim3 grid((a.lay.N + kScoreRows - 1) / kScoreRows, E);
+    const unsigned grid = (unsigned)blocks;
     if (a.lay.dtype == AKV_BF16) score_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(a, h->tab);
     else score_kernel<float><<<grid, kThreads, 0, st>>>(a, h->tab);
     return launched("score");
@@ -251,7 +268,7 @@ static akv_status_t launch_score(akv_handle* h, const EventArgs& a, cudaStream_t
 // General selection: pool-restricted Algorithm 1; the pool's signature rows stay in shared memory
 // when they fit (tile sized to what the device allows).
 template <typename T, bool FLAT>
-static akv_status_t launch_select_pool(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+static akv_status_t launch_select_pool(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
     const int row_bytes = a.lay.d * (int)sizeof(T);
     const PoolSmem fixed = plan_pool_smem(a.lay.N, a.budget, row_bytes, 0);
@@ -261,14 +278,14 @@ static akv_status_t launch_select_pool(akv_handle* h, const EventArgs& a, cudaSt
     if (!a.greedy) tile_rows = 0;
     const PoolSmem sp = plan_pool_smem(a.lay.N, a.budget, row_bytes, tile_rows);
     akv_status_t s = set_smem(select_pool_kernel<T, FLAT>, sp.total);
-    if (s != AKV_OK) return s;
+    if (s != AKV_OK || dry) return s;
     select_pool_kernel<T, FLAT><<<E, kThreads, sp.total, st>>>(a, tile_rows);
     return launched("select_pool");
 }
 template <typename T>
-static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStream_t st) {
-    if (a.flat_sig) return launch_select_pool<float, true>(h, a, st);
-    return launch_select_pool<T, false>(h, a, st);
+static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry) {
+    if (a.flat_sig) return launch_select_pool<float, true>(h, a, st, dry);
+    return launch_select_pool<T, false>(h, a, st, dry);
 }
 
 // Tensor-memory path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.
@@ -276,7 +293,7 @@ static bool tc_path_ok(const EventArgs& a) {
     return a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.flat_sig == nullptr;
 }
 template <bool FUSED>
-static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t st) {
+static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t st, bool dry = false) {
     EventArgs a = a0;
     const int E = a.lay.B * a.lay.L * a.lay.H;
     const TcSmem sp = plan_tc_smem(a.lay.N, a.budget);
@@ -288,6 +305,7 @@ static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t s
     if ((s = set_smem(event_tc_kernel<FUSED>, sp.total)) != AKV_OK) return s;
     CUDA_TRY(cudaFuncSetAttribute(event_tc_kernel<FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                   (int)cudaSharedmemCarveoutMaxShared));
+    if (dry) return AKV_OK;
     event_tc_kernel<FUSED><<<E, kTcThreads, sp.total, st>>>(a, h->tab);
     return launched(FUSED ? "event_tc" : "select_tc");
 }
@@ -296,7 +314,7 @@ static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t s
 // normally stays within 128 rows.
 static bool tri_path_ok(const EventArgs& a) { return tc_path_ok(a) && (a.lay.N <= 128 || a.budget <= 64); }
 template <bool FUSED>
-static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st) {
+static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
     const TriSmem sp = plan_tri_smem(a.lay.N, a.budget);
     if ((int)sp.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "budget %d needs too much shared memory", a.budget);
@@ -304,17 +322,18 @@ static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t s
     if ((s = set_smem(event_tri_kernel<FUSED>, sp.total)) != AKV_OK) return s;
     CUDA_TRY(cudaFuncSetAttribute(event_tri_kernel<FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                   (int)cudaSharedmemCarveoutMaxShared));
+    if (dry) return AKV_OK;
     event_tri_kernel<FUSED><<<E, kTcThreads, sp.total, st>>>(a, h->tab);
     return launched(FUSED ? "event_tri" : "select_tri");
 }
 
-static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st) {
-    if (tri_path_ok(a) && a.V) return launch_tri<false>(h, a, st);
-    if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st);
-    return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st) : launch_select_t<float>(h, a, st);
+static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
+    if (tri_path_ok(a) && a.V) return launch_tri<false>(h, a, st, dry);
+    if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st, dry);
+    return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st, dry) : launch_select_t<float>(h, a, st, dry);
 }
 
-static akv_status_t launch_compact(akv_handle* h, const CompactArgs& a0, cudaStream_t st) {
+static akv_status_t launch_compact(akv_handle* h, const CompactArgs& a0, cudaStream_t st, bool dry = false) {
     CompactArgs a = a0;
     const int E = a.lay.B * a.lay.L * a.lay.H;
     const int rowB = a.lay.d * (a.lay.dtype == AKV_BF16 ? 2 : 4);
@@ -325,11 +344,11 @@ static akv_status_t launch_compact(akv_handle* h, const CompactArgs& a0, cudaStr
     const unsigned bytes = (unsigned)rows * (2 * rowB + 8);
     if (a.lay.dtype == AKV_BF16) {
         akv_status_t s = set_smem(compact_kernel<__nv_bfloat16>, bytes);
-        if (s != AKV_OK) return s;
+        if (s != AKV_OK || dry) return s;
         compact_kernel<__nv_bfloat16><<<E, kThreads, bytes, st>>>(a);
     } else {
         akv_status_t s = set_smem(compact_kernel<float>, bytes);
-        if (s != AKV_OK) return s;
+        if (s != AKV_OK || dry) return s;
         compact_kernel<float><<<E, kThreads, bytes, st>>>(a);
     }
     (void)h;
@@ -339,7 +358,7 @@ static akv_status_t launch_compact(akv_handle* h, const CompactArgs& a0, cudaStr
 // ------------------------------------------------------------------------------------------------
 // entry points
 // ------------------------------------------------------------------------------------------------
-extern "C" akv_status_t alpha_score(akv_handle_t* h, const akv_layout_t* lay, const void* K, const int32_t* pos,
+static akv_status_t alpha_score_impl(akv_handle_t* h, const akv_layout_t* lay, const void* K, const int32_t* pos,
                                     int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand, const float* qstat,
                                     const int32_t* p_ref, const akv_options_t* opt, float* scores, int32_t* status,
                                     void* stream) {
@@ -366,10 +385,16 @@ static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, con
     a.eps = opt->eps;
     a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
     a.no_prune = (opt->flags & AKV_FLAG_NO_PRUNE) ? 1 : 0;
-    if (opt->sig_mode == AKV_SIG_FLAT) {
-        if (!flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat signature mode needs flat_sig");
+    a.starve = (opt->flags & AKV_FLAG_TEST_STARVE_WAIT) ? 1 : 0;
+    a.wait_polls = a.starve ? 64 : kWaitPolls;
+    a.head_budgets = opt->head_budgets;
+    if (opt->sig_mode != AKV_SIG_PER_HEAD) {
+        if (!flat_sig) return fail(AKV_ERR_INVALID_ARG, "shared signature modes need flat_sig");
         if (!aligned16(flat_sig)) return fail(AKV_ERR_ALIGNMENT, "flat_sig is not 16-byte aligned");
         a.flat_sig = flat_sig;
+        const long long nd = (long long)a.lay.N * a.lay.d;
+        a.sig_sb = opt->sig_mode == AKV_SIG_PER_LAYER ? nd * a.lay.L : nd;
+        a.sig_sl = opt->sig_mode == AKV_SIG_PER_LAYER ? nd : 0;
     } else {
         if (flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat_sig given but sig_mode is per-head");
         if (a.greedy && !V) return fail(AKV_ERR_INVALID_ARG, "V must not be NULL in per-head signature mode");
@@ -377,7 +402,7 @@ static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, con
     return AKV_OK;
 }
 
-extern "C" akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, const float* scores, const void* V,
+static akv_status_t alpha_select_impl(akv_handle_t* h, const akv_layout_t* lay, const float* scores, const void* V,
                                      const float* flat_sig, const int32_t* n_cand, int32_t budget,
                                      const akv_options_t* opt, int32_t* idx_sorted, int32_t* pick_order,
                                      float* pick_gain, int32_t* n_kept, int32_t* status, void* stream) {
@@ -402,10 +427,10 @@ extern "C" akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, c
     return launch_select(h, a, (cudaStream_t)stream);
 }
 
-extern "C" akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+static akv_status_t alpha_signature_flat_impl(akv_handle_t* h, const akv_layout_t* lay, const void* V,
                                              const int32_t* n_cand, const akv_options_t* opt, float* flat_sig,
-                                             void* stream) {
-    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_signature_flat: handle is NULL");
+                                             void* stream, int per_layer) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_signature: handle is NULL");
     DevLayout y;
     akv_status_t s = check_layout(lay, &y);
     if (s != AKV_OK) return s;
@@ -416,15 +441,15 @@ extern "C" akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t
     if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
     const int G = pow2_ceil(y.d >> 3) > 32 ? 32 : pow2_ceil(y.d >> 3);
     const long long per_cta = (long long)kWarps * (32 / G);
-    const long long slots = (long long)y.B * y.N;
+    const long long slots = (long long)y.B * (per_layer ? y.L : 1) * y.N;
     const unsigned grid = (unsigned)((slots + per_cta - 1) / per_cta);
     cudaStream_t st = (cudaStream_t)stream;
-    if (y.dtype == AKV_BF16) flat_signature_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig);
-    else flat_signature_kernel<float><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig);
-    return launched("flat_signature");
+    if (y.dtype == AKV_BF16) flat_signature_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig, per_layer);
+    else flat_signature_kernel<float><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig, per_layer);
+    return launched(per_layer ? "layer_signature" : "flat_signature");
 }
 
-extern "C" akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+static akv_status_t kv_compact_impl(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
                                    int64_t psb, int64_t psl, int64_t psh, const int32_t* idx_sorted, int32_t budget,
                                    void* stream) {
     if (!h) return fail(AKV_ERR_INVALID_ARG, "kv_compact: handle is NULL");
@@ -445,7 +470,54 @@ extern "C" akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, voi
     return launch_compact(h, a, (cudaStream_t)stream);
 }
 
-extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+// Which kernels the fused call runs for a shape: the two tensor-memory kernels (bf16, d = 128, N <= 256,
+// per-head signatures), the resident kernel when an event's K and V tiles fit in shared memory, else
+// three launches with the scores in global memory.
+enum EventRoute { ROUTE_TRI, ROUTE_TC, ROUTE_RESIDENT, ROUTE_THREE };
+static EventRoute event_route(const EventArgs& a, int smem_optin) {
+    if (tri_path_ok(a)) return ROUTE_TRI;
+    if (tc_path_ok(a)) return ROUTE_TC;
+    const int es = a.lay.dtype == AKV_BF16 ? 2 : 4;
+    const SmemPlan res = plan_smem(a.lay.N, a.lay.d, es, a.budget, true, true);
+    return (int)res.total <= smem_optin ? ROUTE_RESIDENT : ROUTE_THREE;
+}
+
+extern "C" akv_status_t akv_workspace_bytes(const akv_layout_t* lay, int32_t budget, const akv_options_t* opt, size_t* bytes) {
+    if (!bytes) return fail(AKV_ERR_INVALID_ARG, "akv_workspace_bytes: bytes is NULL");
+    *bytes = 0;
+    EventArgs a;
+    memset(&a, 0, sizeof(a));
+    akv_status_t s = check_layout(lay, &a.lay);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if ((s = check_budget(budget, lay->N)) != AKV_OK) return s;
+    a.budget = budget;
+    a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
+    // only whether shared signatures are in use matters for the route, not where they live
+    a.flat_sig = opt->sig_mode != AKV_SIG_PER_HEAD ? reinterpret_cast<const float*>(bytes) : nullptr;
+    int dev = 0, smem_optin = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (event_route(a, smem_optin) == ROUTE_THREE)
+        *bytes = (size_t)lay->B * lay->L * lay->H * lay->N * sizeof(float);
+    return AKV_OK;
+}
+
+// score -> select -> compact on one stream, the scores passing through a.scores. With `dry` set only
+// the checks of the three launches run (see launch_score).
+static akv_status_t three_launches(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry) {
+    akv_status_t s;
+    EventArgs sa = a;
+    sa.status = nullptr;  // the selection kernel writes the final status word
+    if ((s = launch_score(h, sa, st, dry)) != AKV_OK) return s;
+    if ((s = launch_select(h, a, st, dry)) != AKV_OK) return s;
+    CompactArgs c;
+    memset(&c, 0, sizeof(c));
+    c.lay = a.lay; c.K = a.K; c.V = a.V; c.pos = a.pos; c.idx_sorted = a.idx_sorted; c.budget = a.budget;
+    return launch_compact(h, c, st, dry);
+}
+
+static akv_status_t alpha_compress_event_impl(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
                                              int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand,
                                              const float* qstat, const int32_t* p_ref, const float* flat_sig,
                                              int32_t budget, const akv_options_t* opt, int32_t* idx_sorted,
@@ -474,11 +546,12 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     a.idx_sorted = idx_sorted; a.pick_order = pick_order; a.pick_gain = pick_gain;
     a.scores = scores; a.n_kept = n_kept; a.status = status;
 
-    if (tri_path_ok(a)) return launch_tri<true>(h, a, st);
-    if (tc_path_ok(a)) return launch_tc<true>(h, a, st);
-    const int es = lay->dtype == AKV_BF16 ? 2 : 4;
-    const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
-    if ((int)res.total <= h->smem_optin) {
+    const EventRoute route = event_route(a, h->smem_optin);
+    if (route == ROUTE_TRI) return launch_tri<true>(h, a, st);
+    if (route == ROUTE_TC) return launch_tc<true>(h, a, st);
+    if (route == ROUTE_RESIDENT) {
+        const int es = lay->dtype == AKV_BF16 ? 2 : 4;
+        const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
         const int E = a.lay.B * a.lay.L * a.lay.H;
         if (lay->dtype == AKV_BF16) {
             if ((s = set_smem(event_resident_kernel<__nv_bfloat16>, res.total)) != AKV_OK) return s;
@@ -491,20 +564,14 @@ extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t
     }
     // The event does not fit on chip: score -> select -> compact as three launches, scores held in
     // the caller's buffer or in the handle's scratch.
+    if ((s = three_launches(h, a, st, /*dry=*/true)) != AKV_OK) return s;
     if (!a.scores) {
         void* ws = nullptr;
         const size_t bytes = (size_t)a.lay.B * a.lay.L * a.lay.H * a.lay.N * sizeof(float);
         if ((s = workspace(h, bytes, &ws)) != AKV_OK) return s;
         a.scores = static_cast<float*>(ws);
     }
-    EventArgs sa = a;
-    sa.status = nullptr;  // the selection kernel writes the final status word
-    if ((s = launch_score(h, sa, st)) != AKV_OK) return s;
-    if ((s = launch_select(h, a, st)) != AKV_OK) return s;
-    CompactArgs c;
-    memset(&c, 0, sizeof(c));
-    c.lay = a.lay; c.K = K; c.V = V; c.pos = a.pos; c.idx_sorted = idx_sorted; c.budget = budget;
-    return launch_compact(h, c, st);
+    return three_launches(h, a, st, false);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -531,7 +598,7 @@ static akv_status_t static_scores_address(int device, float** out) {
     return AKV_OK;
 }
 
-extern "C" akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V,
+static akv_status_t alpha_compress_event_static_impl(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V,
                                                     int32_t* pos, int64_t psb, int64_t psl, int64_t psh,
                                                     const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
                                                     const float* flat_sig, int32_t budget, const akv_options_t* opt,
@@ -567,12 +634,57 @@ extern "C" akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_l
     a.scores = scratch; a.n_kept = n_kept; a.status = status;
     // Every score the selection reads (slots below n_cand) is written by the scoring launch of this
     // same call, so nothing left in the array by an earlier call needs clearing.
-    EventArgs sa = a;
-    sa.status = nullptr;  // the selection kernel writes the final status word
-    if ((s = launch_score(h, sa, st)) != AKV_OK) return s;
-    if ((s = launch_select(h, a, st)) != AKV_OK) return s;
-    CompactArgs c;
-    memset(&c, 0, sizeof(c));
-    c.lay = a.lay; c.K = K; c.V = V; c.pos = a.pos; c.idx_sorted = idx_sorted; c.budget = budget;
-    return launch_compact(h, c, st);
+    if ((s = three_launches(h, a, st, /*dry=*/true)) != AKV_OK) return s;
+    return three_launches(h, a, st, false);
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// C entry points: each forwards to its implementation above and leaves a failure's message in the handle.
+// ------------------------------------------------------------------------------------------------
+extern "C" akv_status_t alpha_score(akv_handle_t* h, const akv_layout_t* lay, const void* K, const int32_t* pos,
+                                    int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand, const float* qstat,
+                                    const int32_t* p_ref, const akv_options_t* opt, float* scores, int32_t* status,
+                                    void* stream) {
+    return finish(h, alpha_score_impl(h, lay, K, pos, psb, psl, psh, n_cand, qstat, p_ref, opt, scores, status, stream));
+}
+extern "C" akv_status_t alpha_select(akv_handle_t* h, const akv_layout_t* lay, const float* scores, const void* V,
+                                     const float* flat_sig, const int32_t* n_cand, int32_t budget,
+                                     const akv_options_t* opt, int32_t* idx_sorted, int32_t* pick_order,
+                                     float* pick_gain, int32_t* n_kept, int32_t* status, void* stream) {
+    return finish(h, alpha_select_impl(h, lay, scores, V, flat_sig, n_cand, budget, opt, idx_sorted, pick_order, pick_gain,
+                                       n_kept, status, stream));
+}
+extern "C" akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+                                             const int32_t* n_cand, const akv_options_t* opt, float* flat_sig,
+                                             void* stream) {
+    return finish(h, alpha_signature_flat_impl(h, lay, V, n_cand, opt, flat_sig, stream, 0));
+}
+extern "C" akv_status_t alpha_signature_layer(akv_handle_t* h, const akv_layout_t* lay, const void* V,
+                                              const int32_t* n_cand, const akv_options_t* opt, float* layer_sig,
+                                              void* stream) {
+    return finish(h, alpha_signature_flat_impl(h, lay, V, n_cand, opt, layer_sig, stream, 1));
+}
+extern "C" akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                   int64_t psb, int64_t psl, int64_t psh, const int32_t* idx_sorted, int32_t budget,
+                                   void* stream) {
+    return finish(h, kv_compact_impl(h, lay, K, V, pos, psb, psl, psh, idx_sorted, budget, stream));
+}
+extern "C" akv_status_t alpha_compress_event(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
+                                             int64_t psb, int64_t psl, int64_t psh, const int32_t* n_cand,
+                                             const float* qstat, const int32_t* p_ref, const float* flat_sig,
+                                             int32_t budget, const akv_options_t* opt, int32_t* idx_sorted,
+                                             int32_t* pick_order, float* pick_gain, float* scores, int32_t* n_kept,
+                                             int32_t* status, void* stream) {
+    return finish(h, alpha_compress_event_impl(h, lay, K, V, pos, psb, psl, psh, n_cand, qstat, p_ref, flat_sig, budget, opt,
+                                               idx_sorted, pick_order, pick_gain, scores, n_kept, status, stream));
+}
+extern "C" akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V,
+                                                    int32_t* pos, int64_t psb, int64_t psl, int64_t psh,
+                                                    const int32_t* n_cand, const float* qstat, const int32_t* p_ref,
+                                                    const float* flat_sig, int32_t budget, const akv_options_t* opt,
+                                                    int32_t* idx_sorted, int32_t* pick_order, float* pick_gain,
+                                                    int32_t* n_kept, int32_t* status, void* stream) {
+    return finish(h, alpha_compress_event_static_impl(h, lay, K, V, pos, psb, psl, psh, n_cand, qstat, p_ref, flat_sig, budget,
+                                                      opt, idx_sorted, pick_order, pick_gain, n_kept, status, stream));
 }

@@ -28,7 +28,7 @@ def declared_symbols():
 def test_header_symbols_are_exported(lib):
     syms = declared_symbols()
     assert {"alpha_score", "alpha_select", "kv_compact", "alpha_compress_event", "alpha_signature_flat",
-            "akv_create", "akv_destroy"} <= set(syms)
+            "alpha_signature_layer", "akv_create", "akv_destroy", "akv_last_error", "akv_workspace_bytes"} <= set(syms)
     for s in syms:
         assert hasattr(lib, s), f"{s} declared in alphakv.h but not exported"
     assert set(api.EXPORTS) <= set(syms)
@@ -45,9 +45,20 @@ def test_null_handle_and_bad_arguments_return_codes(lib):
     lay = api.Layout(1, 1, 1, 16, 128, api.AKV_BF16, (2048, 2048, 2048, 128)).c()
     opt = api.Options().c()
     # null handle is rejected before anything else
+    launches = lib.akv_launch_count()
     rc = lib.alpha_score(None, C.byref(lay), None, None, 0, 0, 0, None, None, None, C.byref(opt), None, None, None)
-    assert rc == 1 and b"handle" in lib.akv_last_error()
+    assert rc == 1 and b"handle" in lib.akv_last_error(None)
     rc = lib.kv_compact(None, C.byref(lay), None, None, None, 0, 0, 0, None, 4, None)
     assert rc == 1
     assert lib.akv_status_string(3) == b"budget out of range"
-    assert lib.akv_launch_count() == 0 or lib.akv_launch_count() >= 0
+    assert lib.akv_launch_count() == launches           # a refused call launches nothing
+
+
+def test_workspace_query_validates_before_it_touches_the_device(lib):
+    lay = api.Layout(1, 1, 1, 16, 128, api.AKV_BF16, (2048, 2048, 2048, 128)).c()
+    opt = api.Options().c()
+    out = C.c_size_t(77)
+    assert lib.akv_workspace_bytes(C.byref(lay), 4, C.byref(opt), None) == 1
+    assert lib.akv_workspace_bytes(C.byref(lay), 17, C.byref(opt), C.byref(out)) == 3 and out.value == 0
+    assert b"budget" in lib.akv_last_error(None)
+    assert lib.akv_workspace_bytes(None, 4, C.byref(opt), C.byref(out)) == 1

@@ -50,7 +50,7 @@ def test_c4_large_pool_sampled_events(lam):
     g = run_fused(ev, lam=lam)
     B, L, H, N, d = ev.shape
     rng = np.random.default_rng(4)
-    sample = sorted(rng.choice(B * L * H, size=12, replace=False).tolist())
+    sample = sorted(rng.choice(B * L * H, size=64, replace=False).tolist())
     log = check_all(ev, g, lam, events=sample)
     print("C4 lambda", lam, "near-tie divergences:", log)
     if lam == 0.0:
@@ -64,7 +64,7 @@ def _c5_round(c5, pool_K, pool_V, pos, table, q, lay, opts, sel):
     akv.alpha_compress_event(pool_K, pool_V, pos, q, c5.budget, opts, layout=lay, out=sel)
 
 
-@pytest.mark.parametrize("B,rounds,n_sample", [(4, 3, None), (64, 32, 24)])
+@pytest.mark.parametrize("B,rounds,n_sample", [(4, 3, None), (64, 32, 256)])
 def test_c5_decode_cadence_paged(B, rounds, n_sample):
     c5 = synth.make_c5(B=B, rounds=rounds)
     L, H, N, d, b = c5.L, c5.H, c5.N, c5.d, c5.budget

@@ -24,12 +24,14 @@ def dev(x):
     return akv.to_device(x, "cuda")
 
 
-def run_fused(ev, lam=None, flags=0, n_cand=None, p_ref=True, W=None):
+def run_fused(ev, lam=None, flags=0, n_cand=None, p_ref=True, W=None, budgets=None):
     lam = ev.lam if lam is None else lam
     K, V, pos, q = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat)
     pref = dev(ev.p_ref) if p_ref else None
     nc = None if n_cand is None else dev(np.asarray(n_cand, dtype=np.int32))
-    opts = akv.Options(lam=lam, eps=ev.eps, rope_base=ev.rope_base, future_window=W or ev.future_window, flags=flags)
+    hb = None if budgets is None else dev(np.ascontiguousarray(budgets, dtype=np.int32))
+    opts = akv.Options(lam=lam, eps=ev.eps, rope_base=ev.rope_base, future_window=W or ev.future_window, flags=flags,
+                       head_budgets=hb)
     sel = akv.alpha_compress_event(K, V, pos, q, ev.budget, opts, p_ref=pref, n_cand=nc, want_scores=True)
     torch.cuda.synchronize()
     return dict(K=akv.to_host_bits(K), V=akv.to_host_bits(V), pos=pos.cpu().numpy(), idx=sel.idx_sorted.cpu().numpy(),
@@ -37,7 +39,7 @@ def run_fused(ev, lam=None, flags=0, n_cand=None, p_ref=True, W=None):
                 n_kept=sel.n_kept.cpu().numpy(), status=sel.status.cpu().numpy())
 
 
-def check_all(ev, g, lam, events=None, n_cand=None, p_ref=True, W=None, threads=8):
+def check_all(ev, g, lam, events=None, n_cand=None, p_ref=True, W=None, threads=8, budgets=None):
     B, L, H, N, d = ev.shape
     W = W or ev.future_window
     E = B * L * H
@@ -45,19 +47,20 @@ def check_all(ev, g, lam, events=None, n_cand=None, p_ref=True, W=None, threads=
     ref = None
     if n_cand is None and p_ref and events is None:
         ref = CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lam, W=W, base=ev.rope_base,
-                             eps=ev.eps, threads=threads, want_rows=False)
+                             eps=ev.eps, threads=threads, want_rows=False, budgets=budgets)
     todo = range(E) if events is None else events
     for e in todo:
         b, l, h = e // (L * H), (e // H) % L, e % H
         n = N if n_cand is None else int(n_cand[b])
+        k_e = ev.budget if budgets is None else int(budgets[l][h])
         chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h],
-                        int(ev.p_ref[b]) if p_ref else None, ev.budget, lam,
+                        int(ev.p_ref[b]) if p_ref else None, k_e, lam,
                         g["scores"][b, l, h], g["order"][b, l, h], g["idx"][b, l, h],
                         g["K"][b, l, h], g["V"][b, l, h], g["pos"][b, l, h], W=W, base=ev.rope_base, eps=ev.eps,
                         ref_scores=None if ref is None else ref["scores"][b, l, h],
                         ref_order=None if ref is None else ref["order"][b, l, h], n=n, log=log)
-        assert g["n_kept"][b, l, h] == min(ev.budget, n)
-        assert g["status"][b, l, h] == (2 if n < ev.budget else 0)
+        assert g["n_kept"][b, l, h] == min(k_e, n)
+        assert g["status"][b, l, h] == (2 if n < k_e else 0)
     return log
 
 
@@ -67,8 +70,6 @@ def check_all(ev, g, lam, events=None, n_cand=None, p_ref=True, W=None, threads=
                                         (50, 8, 20), (96, 40, 31)])
 @pytest.mark.parametrize("lam", [0.0, 0.5, 1.5])
 def test_fused_event_small(dtype, N, d, budget, lam):
-    if dtype == synth.F32 and 2 * N * d * 4 > 200_000:
-        pytest.skip("covered by the three-launch path test")
     ev = synth.make_c3(seed=N + d, B=2, L=2, H=3, N=N, budget=budget) if d == 128 else \
         synth.make_plain(2, 2, 3, N, d, budget, lam, dtype=dtype, seed=N + d)
     if d == 128 and dtype == synth.F32:
@@ -219,14 +220,14 @@ def test_flat_signature_eq1_and_selection_with_it():
     opts = akv.Options(lam=0.7, sig_mode=akv.SIG_FLAT)
     sel = akv.alpha_compress_event(K, V, pos, q, 25, opts, p_ref=pref, flat_sig=dev(sig), want_scores=True)
     torch.cuda.synchronize()
-    Kn = akv.to_host_bits(K)
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
     for b in range(2):
         ref_sig = O.signatures_flat(ev.V[b])
         for l in range(3):
             for h in range(2):
                 chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]), 25, 0.7,
                                 sel.scores[b, l, h].cpu().numpy(), sel.pick_order[b, l, h].cpu().numpy(),
-                                sel.idx_sorted[b, l, h].cpu().numpy(), Kn[b, l, h], None, None, sig=ref_sig)
+                                sel.idx_sorted[b, l, h].cpu().numpy(), Kn[b, l, h], Vn[b, l, h], pn[b, l, h], sig=ref_sig)
 
 
 def test_three_launch_path_for_events_that_do_not_fit_on_chip():
@@ -327,3 +328,102 @@ def test_reference_position_behind_some_keys():
     ev.p_ref[:] = np.array([ev.pos[0, 0, 0, 100], ev.pos[0, 0, 0, 0] - 5, ev.pos[0, 0, 0, -1]], dtype=ev.p_ref.dtype)
     g = run_fused(ev)
     check_all(ev, g, ev.lam)
+
+
+# ------------------------------------------------------------------ per-layer signatures, per-head budgets (Section 6)
+@pytest.mark.parametrize("dtype,N,d", [(synth.BF16, 80, 128), (synth.F32, 600, 64)])
+def test_per_layer_signature_mode(dtype, N, d):
+    """Signatures averaged over the heads of one layer: the reduction, and the event that selects with it
+    (resident kernel for the small shape, three launches for the large one)."""
+    ev = synth.make_plain(2, 3, 2, N, d, 25, 0.7, dtype=dtype, seed=27)
+    V = dev(ev.V)
+    sig = akv.alpha_signature_layer(V).cpu().numpy()
+    assert sig.shape == (2, 3, N, d)
+    for b in range(2):
+        for l in range(3):
+            assert np.max(np.abs(sig[b, l] - O.signatures_per_layer(ev.V[b, l]))) < 2e-7
+    K, pos, q, pref = dev(ev.K), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    opts = akv.Options(lam=0.7, sig_mode=akv.SIG_PER_LAYER)
+    sel = akv.alpha_compress_event(K, V, pos, q, 25, opts, p_ref=pref, flat_sig=dev(sig), want_scores=True)
+    torch.cuda.synchronize()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    for b in range(2):
+        for l in range(3):
+            ref_sig = O.signatures_per_layer(ev.V[b, l])
+            for h in range(2):
+                chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]), 25, 0.7,
+                                sel.scores[b, l, h].cpu().numpy(), sel.pick_order[b, l, h].cpu().numpy(),
+                                sel.idx_sorted[b, l, h].cpu().numpy(), Kn[b, l, h], Vn[b, l, h], pn[b, l, h], sig=ref_sig)
+
+
+@pytest.mark.parametrize("maker", ["c3_192", "c2_256", "f32_96", "f32_600"])
+def test_per_head_budgets(maker):
+    """A budget per (layer, head): every kernel family keeps budgets[l, h] rows per event, pads its index rows
+    to the largest budget with -1 and reports the kept count; uniform budgets equal the scalar call."""
+    if maker == "c3_192":
+        ev = synth.make_c3(seed=41, B=2, L=3, H=2, N=192, budget=64)
+    elif maker == "c2_256":
+        ev = synth.make_c2(seed=42, B=2, L=3, H=2)
+    elif maker == "f32_96":
+        ev = synth.make_plain(2, 3, 2, 96, 64, 30, 0.5, dtype=synth.F32, seed=43)
+    else:
+        ev = synth.make_plain(2, 3, 2, 600, 128, 50, 0.5, dtype=synth.F32, seed=44)
+    kmax = ev.budget
+    rng = np.random.default_rng(7)
+    budgets = rng.integers(1, kmax + 1, size=(3, 2)).astype(np.int32)
+    budgets[0, 0], budgets[2, 1] = kmax, 1
+    g = run_fused(ev, budgets=budgets)
+    check_all(ev, g, ev.lam, budgets=budgets)
+    assert int(g["n_kept"].sum()) == 2 * int(budgets.sum())
+    scalar = run_fused(ev)
+    uniform = run_fused(ev, budgets=np.full((3, 2), kmax, dtype=np.int32))
+    for k in ("order", "idx", "K", "V", "pos", "n_kept", "status"):
+        assert np.array_equal(scalar[k], uniform[k]), k
+
+
+# ------------------------------------------------------------------ bounded waits, workspace query, large grids
+@pytest.mark.parametrize("maker", ["tri_192", "tri_96", "tc_256"])
+def test_bounded_wait_runs_out_and_reports_status_3(maker):
+    """With the starve flag no K row is requested and the waits poll only a few times: every wait of the fused
+    tensor-memory kernels runs out with nothing in flight, each event reports status 3, tensor memory is given
+    back (the next, normal call runs) and K, V and positions are left as they were."""
+    if maker == "tri_192":
+        ev = synth.make_c3(seed=51, B=2, L=2, H=2, N=192, budget=64)
+    elif maker == "tri_96":
+        ev = synth.make_c3(seed=52, B=2, L=2, H=2, N=96, budget=40)
+    else:
+        ev = synth.make_c2(seed=53, B=2, L=2, H=2)
+    g = run_fused(ev, flags=akv.FLAG_TEST_STARVE_WAIT)
+    assert np.all(g["status"] == 3)
+    assert np.array_equal(g["K"], ev.K) and np.array_equal(g["V"], ev.V) and np.array_equal(g["pos"], ev.pos)
+    good = run_fused(ev)
+    check_all(ev, good, ev.lam)
+
+
+def test_workspace_query_matches_the_route():
+    bf = akv.Layout(2, 2, 2, 192, 128, akv.api.AKV_BF16, (2 * 2 * 192 * 128, 2 * 192 * 128, 192 * 128, 128))
+    assert akv.workspace_bytes(bf, 64) == 0                                  # on chip, one launch
+    f32_small = akv.Layout(1, 1, 1, 192, 128, akv.api.AKV_F32, (192 * 128,) * 3 + (128,))
+    assert akv.workspace_bytes(f32_small, 64) == 0                           # tiles resident in shared memory
+    f32_big = akv.Layout(1, 2, 2, 600, 128, akv.api.AKV_F32, (4 * 600 * 128, 2 * 600 * 128, 600 * 128, 128))
+    assert akv.workspace_bytes(f32_big, 50) == 1 * 2 * 2 * 600 * 4          # the scores between the launches
+
+
+def test_score_with_more_events_than_a_grid_dimension_holds():
+    """70 000 events: the event index is folded into grid.x, which has room for them."""
+    B, N, d = 70_000, 8, 8
+    rng = np.random.default_rng(61)
+    K = rng.standard_normal((B, 1, 1, N, d)).astype(np.float32)
+    q = rng.standard_normal((1, 1, d)).astype(np.float32)
+    s = akv.alpha_score(dev(K), dev(q), pos=dev(np.arange(N, dtype=np.int32)),
+                        p_ref=dev(np.full(B, N, dtype=np.int32))).cpu().numpy()
+    for b in (0, 1, 65_535, 65_536, B - 1):
+        ref = O.triattention_score(K[b, 0, 0], np.arange(N), q[0, 0], N)
+        chk.check_scores(s[b, 0, 0], ref, chk.score_scale(K[b, 0, 0], q[0, 0], d))
+
+
+def test_report_worst_score_error():
+    """Printed for the record (run last in this file): the worst score error of everything checked so far."""
+    print("worst |err|/|s| where |s| >= 0.1 scale: %.3e; worst |err|/scale: %.3e; scores checked: %d"
+          % (chk.WORST["rel_to_score"], chk.WORST["rel_to_scale"], chk.WORST["n"]))
+    assert chk.WORST["rel_to_score"] <= chk.SCORE_RTOL

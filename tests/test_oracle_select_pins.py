@@ -333,3 +333,52 @@ def test_too_few_finite_scores_still_gives_distinct_indices():
         assert len(set(a.order.tolist())) == 4 and a.order[2:].tolist() == [0, 2]
         oc, _, _, st = CO.select(s, sig, 4, lam)
         assert oc.tolist() == a.order.tolist() and st == O.STATUS_NONFINITE
+
+
+# ----------------------------------------------------------------- per-layer signatures, per-head budgets (Section 6)
+def test_signature_per_layer_is_the_head_mean_and_reduces_to_the_other_modes():
+    rng = np.random.default_rng(41)
+    V = rng.standard_normal((3, 4, 9, 8)).astype(np.float32)           # [L, H, n, d]
+    for l in range(3):
+        sig = O.signatures_per_layer(V[l], 1e-3)
+        u = np.zeros((9, 8))
+        for h in range(4):                                               # the sum of Eq. 1 over this layer's heads only
+            u += V[l, h].astype(np.float64)
+        u /= 4.0
+        assert np.max(np.abs(sig - u / (np.linalg.norm(u, axis=1) + 1e-3)[:, None])) < 1e-15
+        # Eq. 1 over a cache that has only this layer is the same thing
+        assert np.max(np.abs(sig - O.signatures_flat(V[l:l + 1], 1e-3))) < 1e-15
+    # one head per layer: the per-layer signature is the per-head one
+    assert np.max(np.abs(O.signatures_per_layer(V[1, 2:3], 1e-8) - O.signatures_per_head(V[1, 2], 1e-8))) < 1e-15
+
+
+def test_smaller_budget_is_a_prefix_of_the_larger_one():
+    """Eq. 3 defines pick t from the picks before it only, so the selection at budget k' < k is the first k'
+    picks of the selection at budget k: what per-(layer, head) budgets rely on."""
+    s, V = rand_problem(60, 16, 42, corr=0.8)
+    sig = O.signatures_per_head(V)
+    full = O.alpha_select(s, sig, 40, 0.6)
+    for k in (1, 7, 25, 39):
+        part = O.alpha_select(s, sig, k, 0.6)
+        assert np.array_equal(part.order, full.order[:k])
+        assert np.array_equal(CO.select(s, sig, k, 0.6)[0], full.order[:k])
+
+
+def test_event_batch_with_per_head_budgets():
+    ev = synth.make_plain(2, 3, 2, 48, 16, 20, 0.5, dtype=synth.BF16, seed=43)
+    same = CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, 20, 0.5)
+    uni = CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, 20, 0.5, budgets=np.full((3, 2), 20))
+    for k in same:
+        assert np.array_equal(same[k], uni[k]), k                       # uniform budgets = the scalar call
+    bud = np.array([[1, 20], [7, 13], [20, 5]], dtype=np.int32)
+    rag = CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, 20, 0.5, budgets=bud)
+    assert int((rag["idx_sorted"] >= 0).sum()) == 2 * int(bud.sum())    # total kept = sum of the budgets
+    for b in range(2):
+        for l in range(3):
+            for h in range(2):
+                k = int(bud[l, h])
+                r = O.compress_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]), k, 0.5)
+                assert np.array_equal(rag["order"][b, l, h, :k], r.sel.order) and np.all(rag["order"][b, l, h, k:] == -1)
+                assert np.array_equal(rag["idx_sorted"][b, l, h, :k], r.sel.idx_sorted)
+                assert np.array_equal(rag["K"][b, l, h, :k], r.K_new) and np.array_equal(rag["V"][b, l, h, :k], r.V_new)
+                assert np.array_equal(rag["order"][b, l, h, :k], same["order"][b, l, h, :k])

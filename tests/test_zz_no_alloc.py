@@ -1,15 +1,19 @@
 """alpha_compress_event_static: the entry point for callers that may not allocate device memory (a serving
 process whose pool owns the whole device, a decode thread that cannot take cudaMalloc's synchronisation).
 It keeps the intermediate scores in an array inside the library image. Checked here, through the C ABI,
-against alpha_compress_event on the same inputs, twice in a row (the array is shared between calls and keeps
-the earlier call's contents), and for its size limit. Collected last on purpose."""
+against alpha_compress_event on the same inputs and against the CPU oracle, twice in a row (the array is
+shared between calls and keeps the earlier call's contents), for its size limit, and for the claim itself:
+the device's free memory does not move across a call that needs the whole array. Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
 import __graft_entry__ as entry
 import paper_2605_14292_b200 as akv
+from oracle import alpha_oracle as O
 from paper_2605_14292_b200 import synth
+
+import akv_check as chk
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +51,40 @@ def test_static_scratch_entry_matches_the_allocating_one_twice_in_a_row():
         assert np.array_equal(ref["V"][..., :b, :], got["V"][..., :b, :])
         assert np.array_equal(ref["pos"][..., :b], got["pos"][..., :b])
         assert int(got["n_kept"].min()) == b and int(np.abs(got["status"]).max()) == 0
+        # and against the oracle: pick sequence, sorted indices and the compacted rows of every event
+        B, L, H, N, d = ev.shape
+        for bb in range(B):
+            for l in range(L):
+                for h in range(H):
+                    chk.check_event(ev.K[bb, l, h], ev.V[bb, l, h], ev.pos[bb, l, h], ev.qstat[l, h], int(ev.p_ref[bb]),
+                                    b, 0.5, None, got["order"][bb, l, h], got["idx"][bb, l, h], got["K"][bb, l, h],
+                                    got["V"][bb, l, h], got["pos"][bb, l, h])
+
+
+def test_static_scratch_entry_leaves_free_device_memory_unchanged():
+    """A call whose scores fill the whole static array (the allocating entry point would need 4 MiB of scratch
+    for it) with outputs allocated beforehand: free device memory is the same before and after."""
+    small = synth.make_plain(1, 1, 2, 400, 8, 16, 0.5, dtype=synth.F32, seed=33)
+    _run(akv.alpha_compress_event_static, small, 0.5)                      # kernels loaded, symbol address resolved
+    ev = synth.make_plain(8, 4, 4, 8192, 8, 16, 0.5, dtype=synth.F32, seed=34)   # 8*4*4*8192 = 2^20 scores
+    assert ev.n_events * ev.shape[3] == akv.api.STATIC_SCORES_MAX
+    K, V, pos = akv.to_device(ev.K, "cuda"), akv.to_device(ev.V, "cuda"), akv.to_device(ev.pos, "cuda")
+    q, pref = akv.to_device(ev.qstat, "cuda"), akv.to_device(ev.p_ref, "cuda")
+    out = akv.api._alloc_sel(akv.Layout.dense(K), ev.budget, K.device, detail=True)
+    opts = akv.Options(lam=0.5)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    akv.alpha_compress_event_static(K, V, pos, q, ev.budget, opts, p_ref=pref, out=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert int(out.n_kept.min()) == ev.budget and int(out.status.abs().max()) == 0
+    idx, order = out.idx_sorted.cpu().numpy(), out.pick_order.cpu().numpy()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    for e in (0, 37, 127):
+        bb, l, h = e // 16, (e // 4) % 4, e % 4
+        chk.check_event(ev.K[bb, l, h], ev.V[bb, l, h], ev.pos[bb, l, h], ev.qstat[l, h], int(ev.p_ref[bb]), ev.budget, 0.5,
+                        None, order[bb, l, h], idx[bb, l, h], Kn[bb, l, h], Vn[bb, l, h], pn[bb, l, h])
 
 
 def test_static_scratch_entry_rejects_sizes_beyond_its_array():

@@ -85,6 +85,10 @@ typedef struct {
  * waits poll only a few times, so every wait runs out with nothing in flight; each event then
  * reports status 3 and K, V and pos are left as they were. */
 #define AKV_FLAG_TEST_STARVE_WAIT 4u
+/* Testing aid: when an event's positions are an arithmetic progression the fused on-chip kernels turn
+ * the query statistic from row to row by one constant complex factor per frequency instead of taking
+ * every row's sines and cosines afresh; this flag switches that off. Scores agree to rounding. */
+#define AKV_FLAG_NO_CHAIN 8u
 
 typedef struct {
     float lambda;          /* >= 0; 0 takes the top-k branch of Algorithm 1 */

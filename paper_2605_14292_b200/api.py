@@ -23,6 +23,7 @@ SIG_PER_HEAD, SIG_FLAT, SIG_PER_LAYER = 0, 1, 2
 FLAG_FORCE_GREEDY = 1
 FLAG_NO_PRUNE = 2
 FLAG_TEST_STARVE_WAIT = 4
+FLAG_NO_CHAIN = 8
 
 EXPORTS = ("akv_default_options", "akv_create", "akv_destroy", "akv_last_error", "akv_status_string",
            "akv_launch_count", "akv_workspace_bytes", "alpha_score", "alpha_select", "alpha_signature_flat",

@@ -46,6 +46,7 @@ __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget) {
     p.order = o;  o += align16((unsigned)budget * 4);
     p.gain = o;   o += align16((unsigned)budget * 4);
     p.idx = o;    o += align16((unsigned)budget * 4);
+    if (o - p.bypool < 1024u) o = p.bypool + 1024u;  // bypool..idx also hold the folded statistic and the phase steps (1 KB) while scoring
     p.row = p.tile;               // one row of the cosine matrix: plain-dot route only, which leaves the tile unused
     p.sect = o;   o += 256;       // cosine and sine of the 32 sector angles
     p.misc = o;   o += 64;        // mbarriers (K, product, late K rows), tmem base, pool size, block-max scratch
@@ -114,6 +115,75 @@ __device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, c
     }
     return acc2.x + acc2.y;
 }
+
+
+// (cos, sin) of the angle 2 pi ph / 2^32: nearest of the 32 sector angles from the shared-memory table,
+// remainder by the short polynomials of score_lane8
+__device__ __forceinline__ float2 phase_cos_sin(uint32_t ph, const float2* sect) {
+    const float2 e = sect[(ph + 0x04000000u) >> 27];
+    const float w = (float)(int32_t)(ph << 5) * 4.5716245e-11f, z = w * w;
+    const float sw = w * fmaf(z, fmaf(z, 8.3333333e-3f, -0.16666667f), 1.f);
+    const float cw = fmaf(z, fmaf(z, 4.1666667e-2f, -0.5f), 1.f);
+    return make_float2(e.x * cw - e.y * sw, e.y * cw + e.x * sw);
+}
+// bits 32..63 of dist * phi (mod 2^64) for a signed 64-bit distance: the angle dist * theta_f in 2^-32 turns
+__device__ __forceinline__ uint32_t phase_of(long long dist, unsigned long long phi) {
+    const uint32_t dl = (uint32_t)dist, dh = (uint32_t)((unsigned long long)dist >> 32);
+    const uint32_t pl = (uint32_t)phi, ph = (uint32_t)(phi >> 32);
+    return __umulhi(dl, pl) + dl * ph + dh * pl;
+}
+
+// Scoring state of a lane: the folded statistic already turned to the row at hand,
+// G_f = g_f e^{i dist theta_f} for the lane's eight frequencies, so that a row's score is
+// sum_f Re(G_f conj(k_f)); and the turn S_f = e^{-i D theta_f} that takes G from one row of a lane
+// group to its next one when the two rows' positions differ by D (rows 16 slots apart: D = 16 for a
+// cache filled token by token). G is taken afresh (sector table + polynomials) whenever the spacing is
+// not D, and every eighth round in any case: seven chained complex products add less than 4e-8 of the
+// score's scale to the error (fp32 summation of the 64 terms gives 4e-8 by itself).
+struct ChainScore {
+    float2 Gx[4], Gy[4], Sx[4], Sy[4], nSy[4];
+    // S from D (any sign); phitab: phi_f for the lane's frequencies (shared memory)
+    __device__ __forceinline__ void set_step(long long D, const unsigned long long* phitab, const float2* sect) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float2 e = phase_cos_sin(phase_of(-D, phitab[u]), sect);
+            if (u & 1) { Sx[u >> 1].y = e.x; Sy[u >> 1].y = e.y; nSy[u >> 1].y = -e.y; }
+            else { Sx[u >> 1].x = e.x; Sy[u >> 1].x = e.y; nSy[u >> 1].x = -e.y; }
+        }
+    }
+    // G afresh for a row at distance dist (any sign); gtab: folded statistic g_f for the lane's frequencies
+    __device__ __forceinline__ void anchor(long long dist, const float2* gtab, const unsigned long long* phitab,
+                                           const float2* sect) {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float4 g2 = *reinterpret_cast<const float4*>(gtab + 2 * p);       // g of frequencies 2p, 2p + 1
+            const ulonglong2 ph = *reinterpret_cast<const ulonglong2*>(phitab + 2 * p);
+            const float2 ea = phase_cos_sin(phase_of(dist, ph.x), sect), eb = phase_cos_sin(phase_of(dist, ph.y), sect);
+            Gx[p] = make_float2(g2.x * ea.x - g2.y * ea.y, g2.z * eb.x - g2.w * eb.y);
+            Gy[p] = make_float2(g2.x * ea.y + g2.y * ea.x, g2.z * eb.y + g2.w * eb.x);
+        }
+    }
+    __device__ __forceinline__ void advance() {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float2 nx = __ffma2_rn(Gy[p], nSy[p], __fmul2_rn(Gx[p], Sx[p]));
+            const float2 ny = __ffma2_rn(Gy[p], Sx[p], __fmul2_rn(Gx[p], Sy[p]));
+            Gx[p] = nx; Gy[p] = ny;
+        }
+    }
+    // the lane's partial sum of Re(G conj(k)) over its 8 frequencies
+    __device__ __forceinline__ float dot(const uint4& wr, const uint4& wi) const {
+        const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
+        float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            acc2 = __ffma2_rn(Gx[p], make_float2(bf16lo(wre[p]), bf16hi(wre[p])), acc2);
+            acc2 = __ffma2_rn(Gy[p], make_float2(bf16lo(wim[p]), bf16hi(wim[p])), acc2);
+        }
+        return acc2.x + acc2.y;
+    }
+};
+constexpr int kChainRounds = 8;  // rounds between two fresh computations of G
 
 // Per-lane state of the single-warp greedy loop: candidates rho = lane + 32 k, k < CPL.
 template <int CPL>
@@ -316,56 +386,33 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
             spos[j] = p;
             pmax = max(pmax, p);
         }
-        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
-        const int grp = lane >> 3, f0 = (lane & 7) * 8;
-        const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
-        const float inv = rsqrtf((float)kTcD);
-        // folded statistic g_f = c_f z(q)_f / sqrt(d), packed by frequency pairs (f, f+1)
-        float2 gx[4], gy[4], ngx[4];
-        uint32_t phi_lo[8], phi_hi[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const float qr = q[f0 + u] * inv, qi = q[f0 + u + 64] * inv;
-            const float2 c = tab.cw[f0 + u];
-            const float x = c.x * qr - c.y * qi, y = c.x * qi + c.y * qr;
-            if (u & 1) { gx[u >> 1].y = x; gy[u >> 1].y = y; ngx[u >> 1].y = -x; }
-            else { gx[u >> 1].x = x; gy[u >> 1].x = y; ngx[u >> 1].x = -x; }
-            phi_lo[u] = (uint32_t)tab.phi[f0 + u];
-            phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
+        // folded statistic g_f = c_f z(q)_f / sqrt(d) and the frequencies' phase steps, once per event, in
+        // shared memory (storage that the selection uses later)
+        float2* gtab = reinterpret_cast<float2*>(smem + sp.bypool);
+        unsigned long long* phitab = reinterpret_cast<unsigned long long*>(gtab + 64);
+        if (tid < 64) {
+            const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
+            const float inv = rsqrtf((float)kTcD);
+            const float qr = q[tid] * inv, qi = q[tid + 64] * inv;
+            const float2 c = tab.cw[tid];
+            gtab[tid] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+            phitab[tid] = tab.phi[tid];
         }
-        // Distances are measured from `pref`, which is never behind the last key, so that they are
-        // non-negative 32-bit numbers. A reference position behind the last key (rare) is reached by turning
-        // the folded statistic once by the difference: e^{i (p_ref - pos) theta} = e^{i (p_ref - last) theta} e^{i (last - pos) theta}.
-        long long pref = 0;
         if (rotate) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
             if (lane == 0) redi[warp] = pmax;
         }
         __syncthreads();
-        if (rotate) {
-            const long long last = (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3]));
-            pref = a.p_ref ? (long long)a.p_ref[id.b] : last + 1;
-            if (pref < last) {
-                const long long back = pref - last;
-                const uint32_t bl = (uint32_t)back, bh = (uint32_t)((unsigned long long)back >> 32);
-                pref = last;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t ph = __umulhi(bl, phi_lo[u]) + bl * phi_hi[u] + bh * phi_lo[u];
-                    const float2 e = sect[(ph + 0x04000000u) >> 27];
-                    const float w = (float)(int32_t)(ph << 5) * 4.5716245e-11f, z = w * w;
-                    const float sw = w * fmaf(z, fmaf(z, 8.3333333e-3f, -0.16666667f), 1.f);
-                    const float cw = fmaf(z, fmaf(z, 4.1666667e-2f, -0.5f), 1.f);
-                    const float c = e.x * cw - e.y * sw, sn = e.y * cw + e.x * sw;
-                    float& x = (u & 1) ? gx[u >> 1].y : gx[u >> 1].x;
-                    float& y = (u & 1) ? gy[u >> 1].y : gy[u >> 1].x;
-                    float& nx = (u & 1) ? ngx[u >> 1].y : ngx[u >> 1].x;
-                    const float x2 = x * c - y * sn, y2 = x * sn + y * c;
-                    x = x2; y = y2; nx = -x2;
-                }
-            }
-        }
+        long long pref = 0;
+        if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
+        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
+        const int grp = lane >> 3, f0 = (lane & 7) * 8;
+        // spacing of rows 16 slots apart at the newest end of the event: what a token-by-token cache has everywhere
+        const long long D16 = n > 16 ? (long long)spos[n - 1] - (long long)spos[n - 17] : 0;
+        ChainScore cs;
+        cs.set_step(D16, phitab + f0, sect);
+        const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
         // 16 rows per round (4 per warp), in three stretches. Rows from 128 on reuse the slots of rows
         // 0..n_late-1: they are requested after the first stretch, once every warp is past those rows,
         // and awaited before the third. The rounds also run after a timeout (over whatever the tile
@@ -373,18 +420,24 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         auto score_rounds = [&](int round0, int round1) {
             for (int round = round0; round < round1; ++round) {
                 const int j = 16 * round + 4 * warp + grp;
+                const bool live = j < n;
+                // G follows from the previous round's by the constant turn when all four rows of the warp sit
+                // D16 after the rows 16 slots before them
+                bool fresh = (round & (kChainRounds - 1)) == 0 || a.no_chain;
+                if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - 16] == D16);
+                if (fresh) {
+                    if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);
+                } else {
+                    cs.advance();
+                }
                 float acc = 0.f;
-                if (j < n) {
+                if (live) {
                     const unsigned char* krow = tile + (j & (kTriTileRows - 1)) * 256 + (lane & 7) * 16;
-                    const uint4 wr = *reinterpret_cast<const uint4*>(krow);
-                    const uint4 wi = *reinterpret_cast<const uint4*>(krow + 128);
-                    // without positions the distance is 0: sector 0, remainder 0, the rotation is the identity
-                    const uint32_t dist = rotate ? (uint32_t)(pref - (long long)spos[j]) : 0u;
-                    acc = score_lane8<true>(wr, wi, gx, gy, ngx, phi_lo, phi_hi, dist, sect);
+                    acc = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
                 }
 #pragma unroll
                 for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-                if (j < n && (lane & 7) == 0) {
+                if (live && (lane & 7) == 0) {
                     if (a.scores) a.scores[(long long)id.e * N + j] = acc;
                     const bool fin = isfinite(acc);
                     bad |= !fin;
@@ -395,7 +448,6 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
             }
         };
         timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
-        const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
             // first and third stretch share one copy of the loop (the kernel's code should stay small)

@@ -20,6 +20,7 @@ struct EventArgs {
     int greedy;             // 1: run the loop with similarity updates; 0: top-k
     int no_prune;           // 1: keep every candidate in the pool the loop runs over
     int tmem_cols;          // tensor-memory columns the tensor-memory kernel claims per CTA (0: none)
+    int no_chain;           // testing aid: score every row from scratch even when positions are regular
     int starve;             // testing aid: request no K row, so that the bounded waits run out
     int wait_polls;         // polls after which a bounded wait gives up
     int* idx_sorted;

@@ -386,6 +386,7 @@ static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, con
     a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
     a.no_prune = (opt->flags & AKV_FLAG_NO_PRUNE) ? 1 : 0;
     a.starve = (opt->flags & AKV_FLAG_TEST_STARVE_WAIT) ? 1 : 0;
+    a.no_chain = (opt->flags & AKV_FLAG_NO_CHAIN) ? 1 : 0;
     a.wait_polls = a.starve ? 64 : kWaitPolls;
     a.head_budgets = opt->head_budgets;
     if (opt->sig_mode != AKV_SIG_PER_HEAD) {

@@ -472,7 +472,6 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         }
     }
     for (int j = n + tid; j < np4; j += kTcThreads) key[j] = 0u;  // below every real key
-    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
     timeout = __syncthreads_or(timeout);
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
@@ -482,6 +481,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         return;
     }
     bad = __syncthreads_or(bad);
+    // (only now: while scoring, this storage holds the statistic's table, which slower warps may still read)
+    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
 
     // ---- s_(b) by bisection over the score keys, then the pool in slot order (warp 0) -------------
     if (warp == 0) {

@@ -17,7 +17,7 @@
 //   5. Kept rows are written back in place: V from the tile, K and positions re-read (L2) and
 //      staged on chip before the first store.
 #pragma once
-#include "akv_kernels.cuh"
+#include "akv_score_chain.cuh"
 
 namespace akv {
 
@@ -28,7 +28,7 @@ constexpr int kTcCols = 128;     // cosine-matrix columns kept in tensor memory 
 constexpr int kWaitPolls = 1 << 22;
 
 struct TcSmem {
-    unsigned tile, s, key, spos, byrank, rankof, taken, order, gain, idx, slot, misc, total;
+    unsigned tile, s, key, spos, byrank, rankof, taken, order, gain, idx, sect, slot, misc, total;
     int tile_rows;
 };
 // Layout after the 1024-byte aligned base. `key` (ranking) and `r` (reciprocal norms) share storage.
@@ -47,6 +47,8 @@ __host__ __device__ inline TcSmem plan_tc_smem(int N, int budget) {
     p.order = o;  o += align16((unsigned)budget * 4);
     p.gain = o;   o += align16((unsigned)budget * 4);
     p.idx = o;    o += align16((unsigned)budget * 4);
+    if (o - p.byrank < 1024u) o = p.byrank + 1024u;  // byrank..idx also hold the folded statistic and the phase steps (1 KB) while scoring
+    p.sect = o;   o += 256;  // cosine and sine of the 32 sector angles
     p.slot = o;   o += 64;   // 2 x 4 keys of 8 bytes
     p.misc = o;   o += 64;   // mbarriers (2 x 8), tmem base, s_(b), block-max scratch
     p.total = o + 1024;      // room to align the base to 1024 bytes
@@ -146,31 +148,6 @@ __device__ __forceinline__ uint32_t tile_chunk(int rho, int c, uint32_t half_byt
 // the lower original slot.
 __device__ __forceinline__ uint32_t key_low(int orig, int rho) { return ((0xFFFFu - (uint32_t)orig) << 16) | (uint32_t)rho; }
 
-// cos and -sin of 2*pi*(t/2^32) for two phases at once with packed fp32 arithmetic; the octant
-// reduction and the polynomials are those of sincos_phase, so each half gives the same bits.
-__device__ __forceinline__ void sincos_phase2(uint32_t ta, uint32_t tb, float2& cs, float2& nsn) {
-    const uint32_t ua = ta + 0x20000000u, ub = tb + 0x20000000u;
-    const float2 t = make_float2((float)((int)(ua & 0x3FFFFFFFu) - 0x20000000), (float)((int)(ub & 0x3FFFFFFFu) - 0x20000000));
-    const float2 y = __fmul2_rn(t, make_float2(1.862645149230957e-09f, 1.862645149230957e-09f));  // 2^-29
-    const float2 z = __fmul2_rn(y, y);
-    float2 p = __ffma2_rn(z, make_float2(-3.587714997811334e-05f, -3.587714997811334e-05f),
-                          make_float2(0.0024898717780787645f, 0.0024898717780787645f));
-    p = __ffma2_rn(z, p, make_float2(-0.08074536717605851f, -0.08074536717605851f));
-    p = __ffma2_rn(z, p, make_float2(0.7853981525308736f, 0.7853981525308736f));
-    const float2 sp = __fmul2_rn(y, p);
-    float2 c = __ffma2_rn(z, make_float2(-0.0003191315544232772f, -0.0003191315544232772f),
-                          make_float2(0.01585035496683941f, 0.01585035496683941f));
-    c = __ffma2_rn(z, c, make_float2(-0.308424473701413f, -0.308424473701413f));
-    c = __ffma2_rn(z, c, make_float2(1.0f, 1.0f));
-    // quarter turns: bit 30 of u swaps sine and cosine, bit 31 of u (of u + 2^30) flips the sine (cosine)
-    const bool swa = ua & 0x40000000u, swb = ub & 0x40000000u;
-    const uint32_t ca = __float_as_uint(swa ? sp.x : c.x), sa = __float_as_uint(swa ? c.x : sp.x);
-    const uint32_t cb = __float_as_uint(swb ? sp.y : c.y), sb = __float_as_uint(swb ? c.y : sp.y);
-    cs = make_float2(__uint_as_float(ca ^ ((ua + 0x40000000u) & 0x80000000u)),
-                     __uint_as_float(cb ^ ((ub + 0x40000000u) & 0x80000000u)));
-    nsn = make_float2(__uint_as_float(sa ^ (~ua & 0x80000000u)), __uint_as_float(sb ^ (~ub & 0x80000000u)));
-}
-
 // ---- the kernel ------------------------------------------------------------------------------------
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
@@ -197,6 +174,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     float* gain = reinterpret_cast<float*>(smem + sp.gain);
     int* idx = reinterpret_cast<int*>(smem + sp.idx);
     uint2* slot = reinterpret_cast<uint2*>(smem + sp.slot);
+    float2* sect = reinterpret_cast<float2*>(smem + sp.sect);
     const uint32_t barK = smem_u32(smem + sp.misc);
     const uint32_t barM = barK + 8;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 16);
@@ -230,6 +208,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         mbar_init(barM, 1);
         mbar_init_fence();
     }
+    if (FUSED && warp == 1) fill_sector_table(sect, lane);
     __syncthreads();
     uint32_t tbase = 0u;
 
@@ -265,74 +244,45 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
             spos[j] = p;
             pmax = max(pmax, p);
         }
-        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
-        const int grp = lane >> 3, f0 = (lane & 7) * 8;
-        const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
-        const float inv = rsqrtf((float)kTcD);
-        // folded statistic g_f = c_f z(q)_f / sqrt(d), packed by frequency pairs (f, f+1)
-        float2 gx[4], gy[4], ngx[4];
-        uint32_t phi_lo[8], phi_hi[8];
+        // folded statistic and phase steps, once per event, in storage that the selection uses later
+        float2* gtab = reinterpret_cast<float2*>(smem + sp.byrank);
+        unsigned long long* phitab = reinterpret_cast<unsigned long long*>(gtab + 64);
+        fill_statistic_tables(a.qstat + ((long long)id.l * lay.H + id.h) * kTcD, tab, tid, gtab, phitab);
+        if (rotate && !a.p_ref) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const float qr = q[f0 + u] * inv, qi = q[f0 + u + 64] * inv;
-            const float2 c = tab.cw[f0 + u];
-            const float x = c.x * qr - c.y * qi, y = c.x * qi + c.y * qr;
-            if (u & 1) { gx[u >> 1].y = x; gy[u >> 1].y = y; ngx[u >> 1].y = -x; }
-            else { gx[u >> 1].x = x; gy[u >> 1].x = y; ngx[u >> 1].x = -x; }
-            phi_lo[u] = (uint32_t)tab.phi[f0 + u];
-            phi_hi[u] = (uint32_t)(tab.phi[f0 + u] >> 32);
+            for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
+            if (lane == 0) redi[warp] = pmax;
         }
+        __syncthreads();
         long long pref = 0;
-        if (rotate) {
-            if (a.p_ref) {
-                pref = a.p_ref[id.b];
-                __syncthreads();
-            } else {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
-                if (lane == 0) redi[warp] = pmax;
-                __syncthreads();
-                pref = (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
-            }
-        } else {
-            __syncthreads();
-        }
+        if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
+        // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes; the statistic is
+        // carried from one row of the group to the next (see ChainScore)
+        const int grp = lane >> 3, f0 = (lane & 7) * 8;
+        const long long D16 = n > 16 ? (long long)spos[n - 1] - (long long)spos[n - 17] : 0;
+        ChainScore cs;
+        cs.set_step(D16, phitab + f0, sect);
         timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
         if (!timeout) {
-            for (int j0 = 4 * warp; j0 < n; j0 += 4 * (kTcThreads / 32)) {
-                const int j = j0 + grp;
+            const int rounds = (n + 15) >> 4;
+            for (int round = 0; round < rounds; ++round) {
+                const int j = 16 * round + 4 * warp + grp;
+                const bool live = j < n;
+                bool fresh = (round & (kChainRounds - 1)) == 0 || a.no_chain;
+                if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - 16] == D16);
+                if (fresh) {
+                    if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);
+                } else {
+                    cs.advance();
+                }
                 float acc = 0.f;
-                if (j < n) {
-                    const uint4 wr = *reinterpret_cast<const uint4*>(tile + j * 256 + (lane & 7) * 16);
-                    const uint4 wi = *reinterpret_cast<const uint4*>(tile + j * 256 + 128 + (lane & 7) * 16);
-                    const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
-                    const long long dist = pref - (long long)spos[j];
-                    const uint32_t dlo = (uint32_t)dist, dhi = (uint32_t)((unsigned long long)dist >> 32);
-                    float2 acc2 = make_float2(0.f, 0.f);
-#pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        const float2 kre = make_float2(bf16lo(wre[p]), bf16hi(wre[p]));
-                        const float2 kim = make_float2(bf16lo(wim[p]), bf16hi(wim[p]));
-                        // t = g conj(k): real and imaginary part for the two frequencies of the pair
-                        const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
-                        const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
-                        if (rotate) {
-                            // bits 32..63 of dist * phi (mod 2^64)
-                            const uint32_t ta = __umulhi(dlo, phi_lo[2 * p]) + dlo * phi_hi[2 * p] + dhi * phi_lo[2 * p];
-                            const uint32_t tb = __umulhi(dlo, phi_lo[2 * p + 1]) + dlo * phi_hi[2 * p + 1] + dhi * phi_lo[2 * p + 1];
-                            float2 cs, nsn;
-                            sincos_phase2(ta, tb, cs, nsn);
-                            acc2 = __ffma2_rn(tr, cs, acc2);
-                            acc2 = __ffma2_rn(ti, nsn, acc2);
-                        } else {
-                            acc2 = __fadd2_rn(acc2, tr);
-                        }
-                    }
-                    acc = acc2.x + acc2.y;
+                if (live) {
+                    const unsigned char* krow = tile + j * 256 + (lane & 7) * 16;
+                    acc = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
                 }
 #pragma unroll
                 for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-                if (j < n && (lane & 7) == 0) {
+                if (live && (lane & 7) == 0) {
                     if (a.scores) a.scores[(long long)id.e * N + j] = acc;
                     const bool fin = isfinite(acc);
                     bad |= !fin;
@@ -353,7 +303,6 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         }
     }
     for (int j = n + tid; j < np4; j += kTcThreads) key[j] = 0u;  // below every real key
-    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
     timeout = __syncthreads_or(timeout);
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
@@ -361,6 +310,8 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         return;
     }
     bad = __syncthreads_or(bad);
+    // (only now: while scoring, this storage holds the statistic's table, which slower warps may still read)
+    for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
 
     // ---- rank by score (ties to the lower slot) and the pool that can ever be picked ----------------
     int cand[2], rank[2];

@@ -72,119 +72,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 // fall into 32 different banks for a fixed b, and so do consecutive b for a fixed a
 __device__ __forceinline__ int tri_row(int a) { return (a * (a + 1)) >> 1; }
 
-// Score terms of one key row for the 8 frequencies a lane covers, packed by frequency pairs.
-// wr / wi: real and imaginary halves (8 bf16 each); returns the lane's partial sum.
-// The rotation by dist * theta_f is taken in two steps: to the nearest of 32 sector angles, whose
-// cosine and sine come from the shared-memory table `sect`, and by the remainder |w| <= pi/32, whose
-// cosine and sine are short Taylor polynomials (error below 2e-9). With t = g conj(k):
-//   Re(t e^{i(A + w)}) = cos w * Re(t e^{iA}) - sin w * Im(t e^{iA}).
-template <bool ROTATE>
-__device__ __forceinline__ float score_lane8(const uint4& wr, const uint4& wi, const float2 (&gx)[4], const float2 (&gy)[4],
-                                             const float2 (&ngx)[4], const uint32_t (&phi_lo)[8], const uint32_t (&phi_hi)[8],
-                                             uint32_t dist, const float2* sect) {
-    const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
-    float2 acc2 = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int p = 0; p < 4; ++p) {
-        const float2 kre = make_float2(bf16lo(wre[p]), bf16hi(wre[p]));
-        const float2 kim = make_float2(bf16lo(wim[p]), bf16hi(wim[p]));
-        // t = g conj(k): real and imaginary part for the two frequencies of the pair
-        const float2 tr = __ffma2_rn(gx[p], kre, __fmul2_rn(gy[p], kim));
-        if (ROTATE) {
-            const float2 ti = __ffma2_rn(gy[p], kre, __fmul2_rn(ngx[p], kim));
-            // bits 32..63 of dist * phi (mod 2^64): the angle in 2^-32 turns (dist: 32 bits, not negative)
-            const uint32_t ta = __umulhi(dist, phi_lo[2 * p]) + dist * phi_hi[2 * p];
-            const uint32_t tb = __umulhi(dist, phi_lo[2 * p + 1]) + dist * phi_hi[2 * p + 1];
-            // remainder to the nearest sector: the low 27 bits as a signed number (kept scaled by 32)
-            const float2 w = __fmul2_rn(make_float2((float)(int32_t)(ta << 5), (float)(int32_t)(tb << 5)),
-                                        make_float2(4.5716245e-11f, 4.5716245e-11f));  // 2 pi / 2^37
-            const float2 z = __fmul2_rn(w, w);
-            float2 nsl = __ffma2_rn(z, make_float2(-8.3333333e-3f, -8.3333333e-3f), make_float2(0.16666667f, 0.16666667f));
-            nsl = __ffma2_rn(z, nsl, make_float2(-1.f, -1.f));
-            nsl = __fmul2_rn(w, nsl);  // -sin w
-            float2 cl = __ffma2_rn(z, make_float2(4.1666667e-2f, 4.1666667e-2f), make_float2(-0.5f, -0.5f));
-            cl = __ffma2_rn(z, cl, make_float2(1.f, 1.f));  // cos w
-            const float2 ea = sect[(ta + 0x04000000u) >> 27], eb = sect[(tb + 0x04000000u) >> 27];  // (cos A, sin A)
-            const float2 p1 = make_float2(fmaf(tr.x, ea.x, -ti.x * ea.y), fmaf(tr.y, eb.x, -ti.y * eb.y));  // Re(t e^{iA})
-            const float2 p2 = make_float2(fmaf(tr.x, ea.y, ti.x * ea.x), fmaf(tr.y, eb.y, ti.y * eb.x));    // Im(t e^{iA})
-            acc2 = __ffma2_rn(cl, p1, acc2);
-            acc2 = __ffma2_rn(nsl, p2, acc2);
-        } else {
-            acc2 = __fadd2_rn(acc2, tr);
-        }
-    }
-    return acc2.x + acc2.y;
-}
-
-
-// (cos, sin) of the angle 2 pi ph / 2^32: nearest of the 32 sector angles from the shared-memory table,
-// remainder by the short polynomials of score_lane8
-__device__ __forceinline__ float2 phase_cos_sin(uint32_t ph, const float2* sect) {
-    const float2 e = sect[(ph + 0x04000000u) >> 27];
-    const float w = (float)(int32_t)(ph << 5) * 4.5716245e-11f, z = w * w;
-    const float sw = w * fmaf(z, fmaf(z, 8.3333333e-3f, -0.16666667f), 1.f);
-    const float cw = fmaf(z, fmaf(z, 4.1666667e-2f, -0.5f), 1.f);
-    return make_float2(e.x * cw - e.y * sw, e.y * cw + e.x * sw);
-}
-// bits 32..63 of dist * phi (mod 2^64) for a signed 64-bit distance: the angle dist * theta_f in 2^-32 turns
-__device__ __forceinline__ uint32_t phase_of(long long dist, unsigned long long phi) {
-    const uint32_t dl = (uint32_t)dist, dh = (uint32_t)((unsigned long long)dist >> 32);
-    const uint32_t pl = (uint32_t)phi, ph = (uint32_t)(phi >> 32);
-    return __umulhi(dl, pl) + dl * ph + dh * pl;
-}
-
-// Scoring state of a lane: the folded statistic already turned to the row at hand,
-// G_f = g_f e^{i dist theta_f} for the lane's eight frequencies, so that a row's score is
-// sum_f Re(G_f conj(k_f)); and the turn S_f = e^{-i D theta_f} that takes G from one row of a lane
-// group to its next one when the two rows' positions differ by D (rows 16 slots apart: D = 16 for a
-// cache filled token by token). G is taken afresh (sector table + polynomials) whenever the spacing is
-// not D, and every eighth round in any case: seven chained complex products add less than 4e-8 of the
-// score's scale to the error (fp32 summation of the 64 terms gives 4e-8 by itself).
-struct ChainScore {
-    float2 Gx[4], Gy[4], Sx[4], Sy[4], nSy[4];
-    // S from D (any sign); phitab: phi_f for the lane's frequencies (shared memory)
-    __device__ __forceinline__ void set_step(long long D, const unsigned long long* phitab, const float2* sect) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const float2 e = phase_cos_sin(phase_of(-D, phitab[u]), sect);
-            if (u & 1) { Sx[u >> 1].y = e.x; Sy[u >> 1].y = e.y; nSy[u >> 1].y = -e.y; }
-            else { Sx[u >> 1].x = e.x; Sy[u >> 1].x = e.y; nSy[u >> 1].x = -e.y; }
-        }
-    }
-    // G afresh for a row at distance dist (any sign); gtab: folded statistic g_f for the lane's frequencies
-    __device__ __forceinline__ void anchor(long long dist, const float2* gtab, const unsigned long long* phitab,
-                                           const float2* sect) {
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            const float4 g2 = *reinterpret_cast<const float4*>(gtab + 2 * p);       // g of frequencies 2p, 2p + 1
-            const ulonglong2 ph = *reinterpret_cast<const ulonglong2*>(phitab + 2 * p);
-            const float2 ea = phase_cos_sin(phase_of(dist, ph.x), sect), eb = phase_cos_sin(phase_of(dist, ph.y), sect);
-            Gx[p] = make_float2(g2.x * ea.x - g2.y * ea.y, g2.z * eb.x - g2.w * eb.y);
-            Gy[p] = make_float2(g2.x * ea.y + g2.y * ea.x, g2.z * eb.y + g2.w * eb.x);
-        }
-    }
-    __device__ __forceinline__ void advance() {
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            const float2 nx = __ffma2_rn(Gy[p], nSy[p], __fmul2_rn(Gx[p], Sx[p]));
-            const float2 ny = __ffma2_rn(Gy[p], Sx[p], __fmul2_rn(Gx[p], Sy[p]));
-            Gx[p] = nx; Gy[p] = ny;
-        }
-    }
-    // the lane's partial sum of Re(G conj(k)) over its 8 frequencies
-    __device__ __forceinline__ float dot(const uint4& wr, const uint4& wi) const {
-        const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
-        float2 acc2 = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            acc2 = __ffma2_rn(Gx[p], make_float2(bf16lo(wre[p]), bf16hi(wre[p])), acc2);
-            acc2 = __ffma2_rn(Gy[p], make_float2(bf16lo(wim[p]), bf16hi(wim[p])), acc2);
-        }
-        return acc2.x + acc2.y;
-    }
-};
-constexpr int kChainRounds = 8;  // rounds between two fresh computations of G
-
 // Per-lane state of the single-warp greedy loop: candidates rho = lane + 32 k, k < CPL.
 template <int CPL>
 struct GreedyLane {
@@ -294,7 +181,7 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
 template <bool FUSED>
-__global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+__global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const DevLayout& lay = a.lay;
@@ -362,11 +249,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         mbar_init(barL, 1);
         mbar_init_fence();
     }
-    if (FUSED && tid >= 32 && tid < 64) {
-        float sn, cs;
-        sincospif((float)(tid - 32) * 0.0625f, &sn, &cs);  // angle 2 pi h / 32
-        sect[tid - 32] = make_float2(cs, sn);
-    }
+    if (FUSED && warp == 1) fill_sector_table(sect, lane);
     if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), kTcCols);
     tc_fence_before();
     __syncthreads();
@@ -390,14 +273,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         // shared memory (storage that the selection uses later)
         float2* gtab = reinterpret_cast<float2*>(smem + sp.bypool);
         unsigned long long* phitab = reinterpret_cast<unsigned long long*>(gtab + 64);
-        if (tid < 64) {
-            const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
-            const float inv = rsqrtf((float)kTcD);
-            const float qr = q[tid] * inv, qi = q[tid + 64] * inv;
-            const float2 c = tab.cw[tid];
-            gtab[tid] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
-            phitab[tid] = tab.phi[tid];
-        }
+        fill_statistic_tables(a.qstat + ((long long)id.l * lay.H + id.h) * kTcD, tab, tid, gtab, phitab);
         if (rotate) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));

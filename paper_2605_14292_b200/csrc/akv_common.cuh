@@ -53,6 +53,21 @@ __device__ __forceinline__ EventId decode_event(const DevLayout& y, int e) {
     return id;
 }
 
+// ---- per-phase cycle stamps (profiling builds only) -------------------------------------------------
+// Built with -DAKV_PHASE_CLOCKS (python -m paper_2605_14292_b200.build --phase-clocks, a separate library
+// file), thread 0 of every event CTA stores clock64() at the phase boundaries of its kernel into a buffer
+// that akv_debug_phase_buffer() registers: kPhaseSlots values per event. The default build compiles the
+// stamps to nothing.
+constexpr int kPhaseSlots = 16;
+#ifdef AKV_PHASE_CLOCKS
+__device__ long long* g_phase_buf = nullptr;
+__device__ __forceinline__ void phase_stamp(int event, int k) {
+    if (threadIdx.x == 0 && g_phase_buf) g_phase_buf[(long long)event * kPhaseSlots + k] = clock64();
+}
+#else
+__device__ __forceinline__ void phase_stamp(int, int) {}
+#endif
+
 // ---- element access: 4 or 8 consecutive elements widened to fp32 -------------------------------
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

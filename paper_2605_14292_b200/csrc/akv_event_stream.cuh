@@ -1,0 +1,643 @@
+// One-launch event kernel for large candidate pools (bf16, d = 128, per-head signatures, N beyond the
+// 256 rows that the other tensor-memory kernels hold): prefill compression, N = 4096 -> budget 128.
+// One CTA of nine warps per event.
+//
+//   1. K streams through a ring of four 64-row stages (cp.async.bulk + full/empty mbarriers, one
+//      producer warp, eight scoring warps); every row is scored as it lands and only its score stays
+//      on chip. K is read from HBM exactly once.
+//   2. s_(b) by a radix-4 bisection over the score keys (all eight warps), then either the top-k
+//      flags (lambda = 0) or the pool of candidates that can ever be an arg-max of Eq. 2
+//      (s_i >= s_(b) - lambda (1 + slack), see akv_select_pool.cuh), in slot order.
+//   3. Only the pool's V rows are read (about 350 of 4096 at lambda = 0.5), into a K-major,
+//      128-byte-swizzled operand tile in shared memory.
+//   4. Algorithm 1 over the pool, every thread owning up to four candidates (score, norm and running
+//      maximum in registers). After a pick, the cosines of the picked row against the whole pool are
+//      one thin tensor-core product per block of 128 pool rows: tcgen05.mma with the block as one
+//      operand and, as the other, the 16 tile rows around the picked one (no data moves), results
+//      in tensor memory, one tcgen05.ld per candidate. Pool rows beyond the tile (rare) take plain
+//      dot products from global memory; a pool that exceeds even that takes a plain-dot loop.
+//   5. Kept K and V rows are staged on chip and written to slots 0..b-1 of the same buffers.
+#pragma once
+#include "akv_event_tc.cuh"
+
+namespace akv {
+
+constexpr int kStWarps = 8;                        // scoring / selection warps
+constexpr int kStWork = kStWarps * 32;             // their threads
+constexpr int kStThreads = kStWork + 32;           // plus the producer warp
+constexpr int kStStageRows = 64;                   // K rows per ring stage
+constexpr int kStStages = 4;
+constexpr unsigned kStStageBytes = kStStageRows * 256u;
+constexpr unsigned kStRingBytes = kStStages * kStStageBytes;
+constexpr int kStRoundRows = kStWarps * 4;         // rows scored per round (4 per warp)
+constexpr int kStCpl = 4;                          // candidates per thread: pools of up to 1024 rows on the tensor-core route
+constexpr int kStExtra = 256;                      // pool rows beyond the tile that the tensor-core route still takes
+constexpr int kStSpare = 16;                       // tile rows after the last pool row (window of a picked row; scratch row)
+constexpr uint32_t kStTmemCols = 128;              // 8 blocks of 128 pool rows x 16 columns
+
+struct StSmem {
+    unsigned tile, pool, taken, xs, order, gain, idx, gtab, sect, slot, misc, total;
+    unsigned tile_bytes, s, spos, rall, ptaken;  // offsets inside the tile region (valid until the V rows arrive)
+    int cap_rows;                                // pool rows the operand tile holds
+};
+// The tile region holds, in turn: the ring + scores + positions (scoring), the pool's V rows (selection), the
+// kept rows on their way out. The plain-dot route keeps its per-candidate arrays where the V rows would be.
+__host__ __device__ inline StSmem plan_st_smem(int N, int budget, int smem_limit) {
+    StSmem p;
+    const unsigned np = (unsigned)((N + 3) & ~3);
+    unsigned fixed = 0;
+    fixed += align16(np * 2);                     // pool
+    fixed += align16(np);                         // taken
+    fixed += 4u * kStExtra * 4u;                  // xs, xlr, xM, xr: state of the rows beyond the tile
+    fixed += 3 * align16((unsigned)budget * 4);   // order, gain, idx
+    fixed += 1024 + 256 + 256 + 256;              // gtab + phitab, sect, slot, misc
+    fixed += 1024;                                // room to align the base to 1024 bytes
+    const unsigned need = kStRingBytes + 3 * align16(np * 4) + align16(np);  // ring, s, spos, rall, ptaken
+    unsigned tile_bytes = (unsigned)smem_limit > fixed ? ((unsigned)smem_limit - fixed) / 2048u * 2048u : 0u;
+    const unsigned max_tile = (1024u + kStSpare) * 256u;
+    if (tile_bytes > max_tile) tile_bytes = max_tile;
+    // whole blocks of 128 rows (a block's product reads all 128 of its rows), as long as the scoring phase still fits
+    if (tile_bytes / 32768u * 32768u >= need) tile_bytes = tile_bytes / 32768u * 32768u;
+    p.cap_rows = tile_bytes >= need ? (int)(tile_bytes / 256u) - kStSpare : 0;  // 0: the shape does not fit
+    p.tile_bytes = tile_bytes;
+    unsigned o = 0;
+    p.tile = o;   o += tile_bytes;
+    p.pool = o;   o += align16(np * 2);
+    p.taken = o;  o += align16(np);
+    p.xs = o;     o += 4u * kStExtra * 4u;
+    p.order = o;  o += align16((unsigned)budget * 4);
+    p.gain = o;   o += align16((unsigned)budget * 4);
+    p.idx = o;    o += align16((unsigned)budget * 4);
+    p.gtab = o;   o += 1024;   // folded statistic (64 x 8 bytes) and phase steps (64 x 8 bytes)
+    p.sect = o;   o += 256;
+    p.slot = o;   o += 256;    // 2 x 8 arg-max keys of 8 bytes, 2 x 8 norms
+    p.misc = o;   o += 256;    // mbarriers (full, empty, product), tensor-memory base, counters
+    p.total = o + 1024;
+    p.s = kStRingBytes;
+    p.spos = p.s + align16(np * 4);
+    p.rall = p.spos + align16(np * 4);
+    p.ptaken = p.rall + align16(np * 4);
+    return p;
+}
+
+// barrier of the eight work warps (the producer warp has left by the time it is used)
+__device__ __forceinline__ void work_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kStWork) : "memory"); }
+
+// eight bf16 of a row against eight of another, accumulated in fp32 (exact products)
+__device__ __forceinline__ void dot8_bf16(const uint4& a, const uint4& b, float2& acc) {
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        acc = __ffma2_rn(make_float2(bf16lo(aw[i]), bf16hi(aw[i])), make_float2(bf16lo(bw[i]), bf16hi(bw[i])), acc);
+}
+
+__global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab,
+                                                                    int smem_limit) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ int radix_part[2][kStWarps][3];
+    __shared__ int scan_part[2][kStWarps];
+    const DevLayout& lay = a.lay;
+    const EventId id = decode_event(lay, blockIdx.x);
+    const int n = event_n(a, id.b);
+    const int N = lay.N;
+    const int bud = event_budget(a, id);
+    const int picks = min(bud, n);
+    const StSmem sp = plan_st_smem(N, a.budget, smem_limit);
+    unsigned char* tile = smem + sp.tile;
+    float* s = reinterpret_cast<float*>(tile + sp.s);
+    int* spos = reinterpret_cast<int*>(tile + sp.spos);
+    unsigned short* pool = reinterpret_cast<unsigned short*>(smem + sp.pool);
+    unsigned char* taken = smem + sp.taken;
+    float* xs = reinterpret_cast<float*>(smem + sp.xs);  // rows beyond the tile: score, lambda / norm, running maximum, 1 / norm
+    float* xlr = xs + kStExtra;
+    float* xM = xlr + kStExtra;
+    float* xr = xM + kStExtra;
+    int* order = reinterpret_cast<int*>(smem + sp.order);
+    float* gain = reinterpret_cast<float*>(smem + sp.gain);
+    int* idx = reinterpret_cast<int*>(smem + sp.idx);
+    float2* gtab = reinterpret_cast<float2*>(smem + sp.gtab);
+    unsigned long long* phitab = reinterpret_cast<unsigned long long*>(gtab + 64);
+    float2* sect = reinterpret_cast<float2*>(smem + sp.sect);
+    unsigned long long* slot = reinterpret_cast<unsigned long long*>(smem + sp.slot);  // [2][8] keys
+    float* slot_r = reinterpret_cast<float*>(smem + sp.slot + 128);                    // [2][8] norms of the warps' best
+    const uint32_t bar_full = smem_u32(smem + sp.misc);  // 4 barriers
+    const uint32_t bar_empty = bar_full + 32;            // 4 barriers
+    const uint32_t barM = bar_full + 64;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 72);
+    int* cnt = reinterpret_cast<int*>(smem + sp.misc + 80);  // [0] a wait ran out, [1] newest position
+    const uint32_t tile_u32 = smem_u32(tile);
+    const int cap = sp.cap_rows;
+    const uint32_t half_bytes = (uint32_t)(cap + kStSpare) * 128u;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool worker = warp < kStWarps;
+    const bool similarity = a.greedy != 0;
+    const bool dense = lay.page_size == 0;
+    const long long ev_off = dense ? id.b * lay.sb + id.l * lay.sl + id.h * lay.sh : 0;
+    auto rowoff = [&](int j) -> long long {
+        return dense ? ev_off + (long long)j * lay.sn : row_offset(lay, id.b, id.l, id.h, j);
+    };
+    __nv_bfloat16* Kg = reinterpret_cast<__nv_bfloat16*>(a.K);
+    __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
+    const int* gpos = event_pos(a.pos, id);
+    const bool rotate = gpos != nullptr;
+
+    phase_stamp(id.e, 0);  // phases: 0 start, 1 tables + positions, 2 K scored, 3 s_(b), 4 pool / top-k, 5 V rows + norms, 6 picks, 7 outputs, 8 end
+    // ---- set-up: barriers, tables, positions on chip --------------------------------------------------------
+    if (tid == 0) {
+        for (int i = 0; i < kStStages; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, kStWarps);
+        }
+        mbar_init(barM, 1);
+        mbar_init_fence();
+        cnt[0] = 0;
+        cnt[1] = INT_MIN;
+    }
+    if (warp == 1) fill_sector_table(sect, lane);
+    fill_statistic_tables(a.qstat + ((long long)id.l * lay.H + id.h) * kTcD, tab, tid, gtab, phitab);
+    __syncthreads();
+    {
+        int pmax = INT_MIN;
+        for (int j = tid; j < n; j += kStThreads) {
+            const int p = rotate ? gpos[j] : 0;
+            spos[j] = p;
+            pmax = max(pmax, p);
+        }
+        pmax = __reduce_max_sync(0xFFFFFFFFu, pmax);
+        if (lane == 0) atomicMax(&cnt[1], pmax);
+    }
+    __syncthreads();
+    long long pref = 0;
+    if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)cnt[1] + 1;
+
+    phase_stamp(id.e, 1);
+    // ---- K through the ring, scored as it lands ---------------------------------------------------------------
+    const int stages = (n + kStStageRows - 1) / kStStageRows;
+    int bad = 0;
+    if (!worker) {
+        if (lane == 0) {
+            for (int st = 0; st < stages; ++st) {
+                const int sl = st % kStStages;
+                if (st >= kStStages && !mbar_wait_bounded(bar_empty + 8 * sl, (uint32_t)((st / kStStages - 1) & 1), a.wait_polls)) {
+                    atomicExch(&cnt[0], 1);
+                    break;
+                }
+                const int r0 = st * kStStageRows, r1 = min(n, r0 + kStStageRows);
+                mbar_expect_tx(bar_full + 8 * sl, (uint32_t)(r1 - r0) * 256u);
+                // as few copies as the layout allows: the whole stage when its rows are contiguous, whole pages
+                // when pages are, else row by row (starve, a testing aid: none at all, the scoring warps' wait runs out)
+                for (int row = r0; row < r1 && !a.starve;) {
+                    int run = 1;
+                    if (dense && lay.sn == kTcD) run = r1 - row;
+                    else if (!dense && lay.s_page_n == kTcD) run = min(r1 - row, lay.page_size - row % lay.page_size);
+                    bulk_g2s(tile_u32 + (uint32_t)sl * kStStageBytes + (uint32_t)(row - r0) * 256u, Kg + rowoff(row),
+                             (uint32_t)run * 256u, bar_full + 8 * sl);
+                    row += run;
+                }
+            }
+        }
+    } else {
+        const int grp = lane >> 3, f0 = (lane & 7) * 8;
+        // spacing of rows one round (32 slots) apart at the newest end: what a cache filled token by token has everywhere
+        const long long D = n > kStRoundRows ? (long long)spos[n - 1] - (long long)spos[n - 1 - kStRoundRows] : 0;
+        ChainScore cs;
+        cs.set_step(D, phitab + f0, sect);
+        for (int st = 0; st < stages; ++st) {
+            const int sl = st % kStStages;
+            if (!mbar_wait_bounded(bar_full + 8 * sl, (uint32_t)((st / kStStages) & 1), a.wait_polls)) {
+                atomicExch(&cnt[0], 1);
+                break;
+            }
+#pragma unroll 1
+            for (int rr = 0; rr < kStStageRows / kStRoundRows; ++rr) {
+                const int round = st * (kStStageRows / kStRoundRows) + rr;
+                const int j = round * kStRoundRows + 4 * warp + grp;
+                const bool live = j < n;
+                bool fresh = (round & (kChainRounds - 1)) == 0 || a.no_chain;
+                if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - kStRoundRows] == D);
+                if (fresh) {
+                    if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);
+                } else {
+                    cs.advance();
+                }
+                float acc = 0.f;
+                if (live) {
+                    const unsigned char* krow = tile + sl * kStStageBytes + (j - st * kStStageRows) * 256 + (lane & 7) * 16;
+                    acc = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
+                }
+#pragma unroll
+                for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+                if (live && (lane & 7) == 0) {
+                    if (a.scores) a.scores[(long long)id.e * N + j] = acc;
+                    const bool fin = isfinite(acc);
+                    bad |= !fin;
+                    s[j] = fin ? acc : -INFINITY;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_empty + 8 * sl) : "memory");
+        }
+    }
+    __syncthreads();
+    if (cnt[0]) {
+        // a wait ran out: report it, give copies that may still be in flight a bounded chance to land, leave
+        if (tid == 0) {
+            if (a.status) a.status[id.e] = 3;
+            for (int sl = 0; sl < kStStages; ++sl) {
+                mbar_wait_bounded(bar_full + 8 * sl, 0, a.wait_polls);
+                mbar_wait_bounded(bar_full + 8 * sl, 1, a.wait_polls);
+            }
+        }
+        return;
+    }
+    bad = __syncthreads_or(bad);
+    if (!worker) return;  // the producer warp is done; the work warps meet at their own barrier from here on
+
+    phase_stamp(id.e, 2);
+    const int np4 = (N + 3) & ~3;
+    for (int j = tid; j < np4; j += kStWork) taken[j] = 0;
+
+    // ---- s_(b): the picks-th largest score key, two bits per round ---------------------------------------------
+    uint32_t kb = 0u;
+    if (picks > 0) {
+        for (int lo = 30; lo >= 0; lo -= 2) {
+            const uint32_t v1 = kb | (1u << lo), v2 = kb | (2u << lo), v3 = kb | (3u << lo);
+            int c1 = 0, c2 = 0, c3 = 0;
+            for (int j = tid; j < n; j += kStWork) {
+                const uint32_t k = orderable(s[j]);
+                c1 += k >= v1;
+                c2 += k >= v2;
+                c3 += k >= v3;
+            }
+            c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+            c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+            c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+            int (*rp)[3] = radix_part[(lo >> 1) & 1];  // per-warp partial counts, double-buffered by round
+            if (lane == 0) { rp[warp][0] = c1; rp[warp][1] = c2; rp[warp][2] = c3; }
+            work_barrier();
+            int t1 = 0, t2 = 0, t3 = 0;
+#pragma unroll
+            for (int w = 0; w < kStWarps; ++w) { t1 += rp[w][0]; t2 += rp[w][1]; t3 += rp[w][2]; }
+            kb = t3 >= picks ? v3 : (t2 >= picks ? v2 : (t1 >= picks ? v1 : kb));
+        }
+    }
+    phase_stamp(id.e, 3);
+    const float sb = from_orderable(kb);
+
+    // block-wide ordered compaction over the slots: calls emit(j, position) for every flagged slot, in slot
+    // order; returns the number of flagged slots
+    auto ordered_scan = [&](auto&& flag, auto&& emit) -> int {
+        int base = 0;
+        int it = 0;
+        for (int j0 = 0; j0 < n; j0 += kStWork, ++it) {
+            const int j = j0 + tid;
+            const bool in = j < n && flag(j);
+            const uint32_t mask = __ballot_sync(0xFFFFFFFFu, in);
+            int* spart = scan_part[it & 1];
+            if (lane == 0) spart[warp] = __popc(mask);
+            work_barrier();
+            int before = 0, total = 0;
+#pragma unroll
+            for (int w = 0; w < kStWarps; ++w) {
+                before += w < warp ? spart[w] : 0;
+                total += spart[w];
+            }
+            if (in) emit(j, base + before + __popc(mask & ((1u << lane) - 1u)));
+            base += total;
+        }
+        work_barrier();
+        return base;
+    };
+
+    // the winning key of every pick: value in the high word, 0xFFFFFFFF - pool row in the low word
+    // (a thread whose wait on the tensor core ran out offers the all-ones key: every thread then sees it win)
+    auto exchange_best = [&](int t, unsigned long long best, float best_r, float& ri) -> unsigned long long {
+        const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
+        const uint32_t whi = __reduce_max_sync(0xFFFFFFFFu, hi);
+        const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, hi == whi ? lo : 0u);
+        unsigned long long* sl = slot + (t & 1) * kStWarps;
+        float* slr = slot_r + (t & 1) * kStWarps;
+        if (hi == whi && lo == wlo) {  // one lane per warp, unless the warp has no candidate left (all keys 0)
+            sl[warp] = best;
+            slr[warp] = best_r;
+        }
+        work_barrier();
+        unsigned long long top = sl[0];
+        int wtop = 0;
+#pragma unroll
+        for (int w = 1; w < kStWarps; ++w)
+            if (sl[w] > top) { top = sl[w]; wtop = w; }
+        ri = slr[wtop];
+        if (tid == 0) gain[t] = from_orderable((uint32_t)(top >> 32));
+        return top;
+    };
+    auto key_row = [](unsigned long long key) -> int { return (int)(0xFFFFFFFFu - (uint32_t)key); };
+
+    int P = 0;
+    if (!similarity) {
+        // top-k: every key above the picks-th one, and the lowest slots among those equal to it
+        float* ps = reinterpret_cast<float*>(spos);  // positions are no longer needed
+        const int above = ordered_scan([&](int j) { return orderable(s[j]) > kb; }, [&](int j, int) { taken[j] = 1; });
+        ordered_scan([&](int j) { return orderable(s[j]) == kb; }, [&](int j, int pos) { if (pos < picks - above) taken[j] = 1; });
+        // the chosen slots as a pool in slot order, then the pick order: by score, equal scores by slot
+        P = ordered_scan([&](int j) { return taken[j] != 0; }, [&](int j, int pos) { pool[pos] = (unsigned short)j; ps[pos] = s[j]; });
+        for (int rho = tid; rho < P; rho += kStWork) {
+            const uint32_t k = orderable(ps[rho]);
+            int rank = 0;
+            for (int o = 0; o < P; ++o) {
+                const uint32_t ko = orderable(ps[o]);
+                rank += ko > k || (ko == k && o < rho);
+            }
+            order[rank] = pool[rho];
+            gain[rank] = ps[rho];
+        }
+        work_barrier();
+    } else {
+        const float thr = a.no_prune ? -INFINITY : fmaf(-1.001f, a.lam, sb) - 1e-6f * fabsf(sb);  // -inf keeps everyone
+        P = ordered_scan([&](int j) { return !(s[j] < thr); }, [&](int j, int pos) { pool[pos] = (unsigned short)j; });
+
+        phase_stamp(id.e, 4);
+        if (P <= cap + kStExtra && picks > 1) {
+            // ======== tensor-core route ==========================================================================
+            // thread (warp w, lane l) owns pool rows 128 (2 k + w / 4) + 32 (w % 4) + l, k < 4: row r of a block of 128
+            // is lane r of tensor memory, and a warp reads the lanes of its own quarter
+            const int quarter = warp & 3, blk0 = warp >> 2;
+            const int resident = min(P, cap), extras = P - resident;
+            float sv[kStCpl], lr[kStCpl], rr[kStCpl], M[kStCpl];
+            uint32_t alive = 0u;
+#pragma unroll
+            for (int k = 0; k < kStCpl; ++k) {
+                const int rho = 128 * (2 * k + blk0) + 32 * quarter + lane;
+                sv[k] = 0.f; lr[k] = 0.f; rr[k] = 0.f; M[k] = 0.f;
+                if (rho < resident) {
+                    sv[k] = s[pool[rho]];
+                    alive |= 1u << k;
+                }
+            }
+            if (tid < extras) {
+                xs[tid] = s[pool[resident + tid]];
+                xM[tid] = 0.f;
+            }
+            bool xalive = tid < extras;
+            if (warp == 0) tmem_alloc(smem_u32(tmem_holder), kStTmemCols);
+            work_barrier();  // every score has been read: the V rows may land on them
+            for (int x = tid; x < resident * 16; x += kStWork) {
+                const int rho = x >> 4, c = x & 15;
+                cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(pool[rho]) + c * 8);
+            }
+            cp_async_wait_all();
+            fence_proxy_async();
+            tc_fence_before();
+            work_barrier();
+            tc_fence_after();
+            const uint32_t tbase = *tmem_holder;
+            // reciprocal norms (Eq. 1)
+#pragma unroll
+            for (int k = 0; k < kStCpl; ++k) {
+                if (alive & (1u << k)) {
+                    const int rho = 128 * (2 * k + blk0) + 32 * quarter + lane;
+                    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll 4
+                    for (int c = 0; c < 16; ++c) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(tile + tile_chunk(rho, c, half_bytes));
+                        dot8_bf16(v, v, acc);
+                    }
+                    rr[k] = 1.f / (sqrtf(acc.x + acc.y) + a.eps);
+                    lr[k] = a.lam * rr[k];
+                }
+            }
+            if (xalive) {
+                const __nv_bfloat16* vrow = Vg + rowoff(pool[resident + tid]);
+                float2 acc = make_float2(0.f, 0.f);
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(vrow + c * 8);
+                    dot8_bf16(v, v, acc);
+                }
+                xr[tid] = 1.f / (sqrtf(acc.x + acc.y) + a.eps);
+                xlr[tid] = a.lam * xr[tid];
+            }
+            phase_stamp(id.e, 5);
+            const int nblk = (resident + 127) >> 7;
+            const uint32_t idesc = umma_idesc_bf16(128, 16);
+            int timeout = 0;
+            uint32_t mround = 0;
+            for (int t = 0; t < picks; ++t) {
+                // Eq. 2 for the candidates still competing, Eq. 3's arg-max (ties to the lower pool row = lower slot)
+                unsigned long long best = 0ull;
+                float best_r = 0.f;
+#pragma unroll
+                for (int k = 0; k < kStCpl; ++k) {
+                    if (alive & (1u << k)) {
+                        const int rho = 128 * (2 * k + blk0) + 32 * quarter + lane;
+                        const unsigned long long key = ((unsigned long long)orderable(fmaf(-lr[k], M[k], sv[k])) << 32) |
+                                                       (unsigned long long)(0xFFFFFFFFu - (uint32_t)rho);
+                        if (key > best) { best = key; best_r = rr[k]; }
+                    }
+                }
+                if (xalive) {
+                    const unsigned long long key = ((unsigned long long)orderable(fmaf(-xlr[tid], xM[tid], xs[tid])) << 32) |
+                                                   (unsigned long long)(0xFFFFFFFFu - (uint32_t)(resident + tid));
+                    if (key > best) { best = key; best_r = xr[tid]; }
+                }
+                if (timeout) best = ~0ull;
+                float ri;
+                const unsigned long long top = exchange_best(t, best, best_r, ri);
+                if (top == ~0ull) {  // some thread's wait ran out in the previous pick
+                    timeout = 1;
+                    break;
+                }
+                const int irho = key_row(top);
+                if (tid == 0) order[t] = pool[irho];
+#pragma unroll
+                for (int k = 0; k < kStCpl; ++k)
+                    if (128 * (2 * k + blk0) + 32 * quarter + lane == irho) alive &= ~(1u << k);
+                if (resident + tid == irho) xalive = false;
+                if (t + 1 == picks) break;
+                // cosines of the picked row against the pool: per block of 128 rows, block x (16 tile rows around the picked one)^T
+                int base = irho & ~7;
+                if (irho >= resident) {
+                    // the picked row lies beyond the tile: it becomes the scratch row after the last pool row
+                    base = cap;
+                    if (tid < 16) cp_async16(tile_u32 + tile_chunk(cap, tid, half_bytes), Vg + rowoff(pool[irho]) + tid * 8);
+                    cp_async_wait_all();
+                    fence_proxy_async();
+                    work_barrier();
+                }
+                const int col = irho >= resident ? 0 : irho - base;
+                if (tid == 0) {
+                    tc_fence_after();
+                    for (int blk = 0; blk < nblk; ++blk) {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
+                            umma_bf16(tbase + (uint32_t)(16 * blk), umma_desc_sw128(tile_u32 + (uint32_t)blk * 16384u + koff),
+                                      umma_desc_sw128(tile_u32 + (uint32_t)base * 128u + koff), idesc, kk > 0 ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(barM);
+                }
+                // rows beyond the tile: plain dot products, both rows read in place, while the tensor core works
+                if (xalive) {
+                    const __nv_bfloat16* vrow = Vg + rowoff(pool[resident + tid]);
+                    const __nv_bfloat16* vpick = Vg + rowoff(pool[irho]);
+                    float2 acc = make_float2(0.f, 0.f);
+                    for (int c = 0; c < 16; ++c)
+                        dot8_bf16(*reinterpret_cast<const uint4*>(vrow + c * 8), *reinterpret_cast<const uint4*>(vpick + c * 8), acc);
+                    xM[tid] = fmaxf(xM[tid], ri * (acc.x + acc.y));
+                }
+                if (!mbar_wait_bounded(barM, mround & 1u, a.wait_polls)) timeout = 1;  // offered to everyone at the next exchange
+                ++mround;
+                tc_fence_after();
+                {
+                    // tcgen05.ld is a warp-wide instruction: every lane issues it, for every block the pool has
+                    // (a warp-uniform test); what a retired candidate reads is not used
+                    float dv[kStCpl];
+#pragma unroll
+                    for (int k = 0; k < kStCpl; ++k)
+                        dv[k] = (2 * k + blk0 < nblk)
+                                    ? tmem_ld1(tbase + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(16 * (2 * k + blk0) + col))
+                                    : 0.f;
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < kStCpl; ++k)
+                        if (alive & (1u << k)) M[k] = fmaxf(M[k], ri * dv[k]);
+                }
+                tc_fence_before();
+            }
+            tc_fence_before();
+            work_barrier();
+            if (warp == 0) tmem_dealloc(tbase, kStTmemCols);
+            if (timeout) {  // uniform: it comes out of an exchange
+                if (tid == 0 && a.status) a.status[id.e] = 3;
+                return;
+            }
+        } else {
+            // ======== plain-dot route: any pool size; V rows read in place, state where the V rows would be ======
+            float* ps = reinterpret_cast<float*>(spos);
+            float* m = s;
+            float* r = reinterpret_cast<float*>(tile + sp.rall);
+            unsigned char* ptaken = tile + sp.ptaken;
+            for (int rho = tid; rho < P; rho += kStWork) ps[rho] = s[pool[rho]];
+            work_barrier();  // s is dead: every pool score sits in ps
+            for (int rho = tid; rho < P; rho += kStWork) {
+                m[rho] = 0.f;
+                ptaken[rho] = 0;
+            }
+            // Work items: (pool row, half) with the halves taking alternate 16-byte chunks; neighbouring lanes hold
+            // the two halves of one row and combine them with one shuffle.
+            const int items = 2 * P, items_up = (items + 31) & ~31;
+            auto vchunk = [&](int rho, int c) -> uint4 { return *reinterpret_cast<const uint4*>(Vg + rowoff(pool[rho]) + c * 8); };
+            for (int i = tid; i < items_up; i += kStWork) {
+                const int rho = i >> 1, half = i & 1;
+                float2 acc = make_float2(0.f, 0.f);
+                if (rho < P) {
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) {
+                        const uint4 v = vchunk(rho, 2 * cc + half);
+                        dot8_bf16(v, v, acc);
+                    }
+                }
+                float ss = acc.x + acc.y;
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+                if (rho < P && half == 0) r[rho] = 1.f / (sqrtf(ss) + a.eps);
+            }
+            work_barrier();
+            // Pass t folds the cosines of pick t - 1 into every candidate's running maximum and, in the same sweep,
+            // finds the arg-max of Eq. 2 for pick t. The first pass (no pick yet) is the plain arg-max of the scores.
+            int irho = -1;
+            float ri = 0.f;
+            for (int t = 0; t < picks; ++t) {
+                unsigned long long best = 0ull;
+                float best_r = 0.f;
+                for (int i = tid; i < items_up; i += kStWork) {
+                    const int rho = i >> 1, half = i & 1;
+                    const bool live = rho < P && !ptaken[rho] && rho != irho;  // (the last pick's flag may not be visible yet)
+                    float dotv = 0.f;
+                    if (irho >= 0) {
+                        float2 acc = make_float2(0.f, 0.f);
+                        if (live) {
+#pragma unroll
+                            for (int cc = 0; cc < 8; ++cc) dot8_bf16(vchunk(rho, 2 * cc + half), vchunk(irho, 2 * cc + half), acc);
+                        }
+                        dotv = acc.x + acc.y;
+                        dotv += __shfl_xor_sync(0xFFFFFFFFu, dotv, 1);
+                    }
+                    if (live && half == 0) {
+                        float mm = m[rho];
+                        if (irho >= 0) {
+                            mm = fmaxf(mm, dotv * (ri * r[rho]));
+                            m[rho] = mm;
+                        }
+                        const unsigned long long key = ((unsigned long long)orderable(fmaf(-a.lam, mm, ps[rho])) << 32) |
+                                                       (unsigned long long)(0xFFFFFFFFu - (uint32_t)rho);
+                        if (key > best) { best = key; best_r = r[rho]; }
+                    }
+                }
+                irho = key_row(exchange_best(t, best, best_r, ri));
+                if (tid == 0) {
+                    order[t] = pool[irho];
+                    ptaken[irho] = 1;
+                }
+            }
+        }
+        work_barrier();
+        for (int t = tid; t < picks; t += kStWork) taken[order[t]] = 1;
+        work_barrier();
+    }
+
+    phase_stamp(id.e, 6);
+    // ---- sort(S) and outputs -------------------------------------------------------------------------
+    if (warp == 0) {
+        int off = 0;
+        for (int base = 0; base < n; base += 32) {
+            const int j = base + lane;
+            const bool f = j < n && taken[j];
+            const unsigned mask = __ballot_sync(0xFFFFFFFFu, f);
+            if (f) idx[off + __popc(mask & ((1u << lane) - 1u))] = j;
+            off += __popc(mask);
+        }
+        for (int t = off + lane; t < a.budget; t += 32) idx[t] = -1;
+    }
+    work_barrier();
+    const long long ob = (long long)id.e * a.budget;
+    for (int t = tid; t < a.budget; t += kStWork) {
+        a.idx_sorted[ob + t] = idx[t];
+        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
+        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
+    }
+    if (tid == 0) {
+        if (a.n_kept) a.n_kept[id.e] = picks;
+        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
+    }
+
+    phase_stamp(id.e, 7);
+    // ---- compaction in place: every kept row of a chunk is on chip before the chunk's first store --------
+    // (a chunk's destinations [c0, c1) can only be sources of the same or of later chunks: idx is ascending
+    // and idx[t] >= t; later chunks' sources lie at or beyond their own destinations)
+    int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
+    const int chunk = (int)(kStRingBytes / 512u);  // rows of K and V together that the ring region holds
+    for (int c0 = 0; c0 < picks; c0 += chunk) {
+        const int cn = min(chunk, picks - c0);
+        work_barrier();
+        for (int x = tid; x < cn * 16; x += kStWork) {
+            const long long off = rowoff(idx[c0 + (x >> 4)]) + (x & 15) * 8;
+            cp_async16(tile_u32 + (uint32_t)x * 16u, Kg + off);
+            cp_async16(tile_u32 + (uint32_t)(chunk * 256) + (uint32_t)x * 16u, Vg + off);
+        }
+        int pv = 0;
+        if (wpos && tid < cn) pv = gpos[idx[c0 + tid]];
+        cp_async_wait_all();
+        work_barrier();
+        for (int x = tid; x < cn * 16; x += kStWork) {
+            const long long off = rowoff(c0 + (x >> 4)) + (x & 15) * 8;
+            *reinterpret_cast<uint4*>(Kg + off) = *reinterpret_cast<const uint4*>(tile + x * 16);
+            *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(tile + chunk * 256 + x * 16);
+        }
+        if (wpos && tid < cn) wpos[c0 + tid] = pv;
+    }
+    phase_stamp(id.e, 8);
+}
+
+}  // namespace akv

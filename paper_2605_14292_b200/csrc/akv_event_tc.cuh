@@ -75,10 +75,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `polls` polls instead of spinning for ever.
+// Bounded wait: gives up after `polls` polls, or after kWaitNs of wall-clock time (a poll may itself
+// suspend the thread for a while, so a poll count alone can stand for minutes), instead of spinning for ever.
+constexpr unsigned long long kWaitNs = 200ull * 1000ull * 1000ull;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int polls) {
-    for (int it = 0; it < polls; ++it)
+    unsigned long long t0 = 0ull;
+    for (int it = 0; it < polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 63) {
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0ull) t0 = now;
+            else if (now - t0 > kWaitNs) return false;
+        }
+    }
     return false;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -212,6 +222,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     __syncthreads();
     uint32_t tbase = 0u;
 
+    phase_stamp(id.e, 0);  // phases: 0 start, 1 K scored, 2 ranks + pool, 3 V operand + tensor memory, 4 product + norms, 5 picks, 6 outputs, 7 end
     // ---- scores ---------------------------------------------------------------------------------
     int bad = 0;
     int timeout = 0;
@@ -313,6 +324,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     // (only now: while scoring, this storage holds the statistic's table, which slower warps may still read)
     for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
 
+    phase_stamp(id.e, 1);
     // ---- rank by score (ties to the lower slot) and the pool that can ever be picked ----------------
     int cand[2], rank[2];
     float sc[2];
@@ -370,6 +382,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     const int cstride = two ? (int)(tcols >> 1) : (int)tcols;
     const int ncols = min((P + 15) & ~15, min(cstride, 128));
 
+    phase_stamp(id.e, 2);
     // ---- V rows of the pool, in rank order, as the swizzled operand tile ---------------------------
     const int vrows = (similarity || FUSED) ? P : 0;
     for (int x = tid; x < vrows * 16; x += kTcThreads) {
@@ -385,6 +398,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     tc_fence_after();
     if (use_tc) tbase = *tmem_holder;
 
+    phase_stamp(id.e, 3);
     const bool do_mma = use_tc && picks > 1;
     if (do_mma && tid == 0) {
         tc_fence_after();
@@ -438,6 +452,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         return;
     }
 
+    phase_stamp(id.e, 4);
     // ---- Algorithm 1 ----------------------------------------------------------------------------------
     const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);
     if (!similarity) {
@@ -549,6 +564,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         __syncthreads();
     }
 
+    phase_stamp(id.e, 5);
     // ---- sort(S) and outputs -------------------------------------------------------------------------
     ordered_indices(n, a.budget, taken, idx);
     __syncthreads();
@@ -564,6 +580,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     }
     if (!FUSED) return;
 
+    phase_stamp(id.e, 6);
     // ---- compaction in place ----------------------------------------------------------------------
     // Every kept K row and position is on chip (registers for up to 64 rows, else the tile) before
     // the first store: a destination slot can be another kept row's source.
@@ -611,6 +628,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
     }
     if (wpos)
         for (int t = tid; t < picks; t += kTcThreads) wpos[t] = spos[idx[t]];
+    phase_stamp(id.e, 7);
 }
 
 }  // namespace akv

@@ -226,6 +226,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     __nv_bfloat16* Kg = reinterpret_cast<__nv_bfloat16*>(a.K);
     __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
 
+    phase_stamp(id.e, 0);  // phases: 0 start, 1 tensor memory claimed, 2 K scored, 3 pool, 4 V operand, 5 product, 6 triangle, 7 picks, 8 outputs, 9 end
     // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
     // next CTA of this kernel only after that, so a late allocation would serialise the CTAs.
     const bool use_tc = similarity;
@@ -256,6 +257,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     tc_fence_after();
     const uint32_t tbase = use_tc ? *tmem_holder : 0u;
 
+    phase_stamp(id.e, 1);
     // ---- scores ---------------------------------------------------------------------------------
     int bad = 0;
     int timeout = 0;
@@ -360,6 +362,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     // (only now: while scoring, this storage holds the statistic's table, which slower warps may still read)
     for (int j = tid; j < np4; j += kTcThreads) taken[j] = 0;
 
+    phase_stamp(id.e, 2);
     // ---- s_(b) by bisection over the score keys, then the pool in slot order (warp 0) -------------
     if (warp == 0) {
         uint32_t kk[8];
@@ -407,6 +410,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     const bool fast = similarity && P <= kTriMaxPool && picks > 1;
     const bool slow = similarity && P > kTriMaxPool;
 
+    phase_stamp(id.e, 3);
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
     if (similarity && !slow) {
         // thread -> 16-byte column c of rows r0, r0 + 8, ...: the swizzle term (c ^ row) & 7 is the same for
@@ -425,6 +429,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
         fence_proxy_async();
         __syncthreads();
     }
+    phase_stamp(id.e, 4);
     if (fast) {
         if (tid == 0) {
             tc_fence_after();
@@ -445,6 +450,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
         if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
         return;
     }
+    phase_stamp(id.e, 5);
     if (fast) {
         // lower triangle -> shared memory; row rho = 32 warp + lane needs columns 0..rho
         const int rho = 32 * warp + lane;
@@ -493,6 +499,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     __syncthreads();
     if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
 
+    phase_stamp(id.e, 6);
     // ---- Algorithm 1 in warp 0 -------------------------------------------------------------------------
     // The winning key of every pick is parked in gain[] and its pool row in order[]; both are decoded
     // after the loop.
@@ -549,6 +556,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     }
     __syncthreads();
 
+    phase_stamp(id.e, 7);
     // ---- sort(S) and outputs -------------------------------------------------------------------------
     ordered_indices(n, a.budget, taken, idx);
     __syncthreads();
@@ -564,6 +572,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     }
     if (!FUSED) return;
 
+    phase_stamp(id.e, 8);
     // ---- compaction in place ----------------------------------------------------------------------
     // Every kept K and V row and position is on chip before the first store: a destination slot can be
     // another kept row's source. Up to 64 rows: K in registers, V through the (by now free) tile by
@@ -602,6 +611,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     }
     if (wpos)
         for (int t = tid; t < picks; t += kTcThreads) wpos[t] = spos[idx[t]];
+    phase_stamp(id.e, 9);
 }
 
 }  // namespace akv

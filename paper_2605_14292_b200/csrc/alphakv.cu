@@ -9,6 +9,7 @@
 #include <cstring>
 
 #include "akv_event_tri.cuh"
+#include "akv_event_stream.cuh"
 #include "akv_select_pool.cuh"
 
 using namespace akv;
@@ -474,10 +475,18 @@ static akv_status_t kv_compact_impl(akv_handle_t* h, const akv_layout_t* lay, vo
 // Which kernels the fused call runs for a shape: the two tensor-memory kernels (bf16, d = 128, N <= 256,
 // per-head signatures), the resident kernel when an event's K and V tiles fit in shared memory, else
 // three launches with the scores in global memory.
-enum EventRoute { ROUTE_TRI, ROUTE_TC, ROUTE_RESIDENT, ROUTE_THREE };
+enum EventRoute { ROUTE_TRI, ROUTE_TC, ROUTE_STREAM, ROUTE_RESIDENT, ROUTE_THREE };
+// shared memory the streaming kernel may plan with: what the device allows minus its static arrays
+static int stream_smem_limit(int smem_optin) { return smem_optin - 1024; }
+static bool stream_path_ok(const EventArgs& a, int smem_optin) {
+    if (!(a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N > kTcMaxN && a.lay.N <= 65535 && a.flat_sig == nullptr)) return false;
+    const StSmem sp = plan_st_smem(a.lay.N, a.budget, stream_smem_limit(smem_optin));
+    return sp.cap_rows > 0 && (int)sp.total <= stream_smem_limit(smem_optin);
+}
 static EventRoute event_route(const EventArgs& a, int smem_optin) {
     if (tri_path_ok(a)) return ROUTE_TRI;
     if (tc_path_ok(a)) return ROUTE_TC;
+    if (stream_path_ok(a, smem_optin)) return ROUTE_STREAM;
     const int es = a.lay.dtype == AKV_BF16 ? 2 : 4;
     const SmemPlan res = plan_smem(a.lay.N, a.lay.d, es, a.budget, true, true);
     return (int)res.total <= smem_optin ? ROUTE_RESIDENT : ROUTE_THREE;
@@ -550,6 +559,13 @@ static akv_status_t alpha_compress_event_impl(akv_handle_t* h, const akv_layout_
     const EventRoute route = event_route(a, h->smem_optin);
     if (route == ROUTE_TRI) return launch_tri<true>(h, a, st);
     if (route == ROUTE_TC) return launch_tc<true>(h, a, st);
+    if (route == ROUTE_STREAM) {
+        const int limit = stream_smem_limit(h->smem_optin);
+        const StSmem sp = plan_st_smem(a.lay.N, a.budget, limit);
+        if ((s = set_smem(event_stream_kernel, sp.total)) != AKV_OK) return s;
+        event_stream_kernel<<<a.lay.B * a.lay.L * a.lay.H, kStThreads, sp.total, st>>>(a, h->tab, limit);
+        return launched("event_stream");
+    }
     if (route == ROUTE_RESIDENT) {
         const int es = lay->dtype == AKV_BF16 ? 2 : 4;
         const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
@@ -689,3 +705,12 @@ extern "C" akv_status_t alpha_compress_event_static(akv_handle_t* h, const akv_l
     return finish(h, alpha_compress_event_static_impl(h, lay, K, V, pos, psb, psl, psh, n_cand, qstat, p_ref, flat_sig, budget,
                                                       opt, idx_sorted, pick_order, pick_gain, n_kept, status, stream));
 }
+
+#ifdef AKV_PHASE_CLOCKS
+// Profiling builds only: registers a device buffer of kPhaseSlots int64 per event for the kernels' phase
+// stamps (NULL switches them off again).
+extern "C" int akv_debug_phase_buffer(long long* device_buffer) {
+    return (int)cudaMemcpyToSymbol(akv::g_phase_buf, &device_buffer, sizeof(device_buffer));
+}
+extern "C" int akv_debug_phase_slots(void) { return akv::kPhaseSlots; }
+#endif

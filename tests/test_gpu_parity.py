@@ -407,6 +407,8 @@ def test_workspace_query_matches_the_route():
     assert akv.workspace_bytes(f32_small, 64) == 0                           # tiles resident in shared memory
     f32_big = akv.Layout(1, 2, 2, 600, 128, akv.api.AKV_F32, (4 * 600 * 128, 2 * 600 * 128, 600 * 128, 128))
     assert akv.workspace_bytes(f32_big, 50) == 1 * 2 * 2 * 600 * 4          # the scores between the launches
+    bf_big = akv.Layout(1, 2, 2, 4096, 128, akv.api.AKV_BF16, (4 * 4096 * 128, 2 * 4096 * 128, 4096 * 128, 128))
+    assert akv.workspace_bytes(bf_big, 128) == 0                             # streaming kernel, scores stay on chip
 
 
 def test_score_with_more_events_than_a_grid_dimension_holds():
@@ -420,6 +422,77 @@ def test_score_with_more_events_than_a_grid_dimension_holds():
     for b in (0, 1, 65_535, 65_536, B - 1):
         ref = O.triattention_score(K[b, 0, 0], np.arange(N), q[0, 0], N)
         chk.check_scores(s[b, 0, 0], ref, chk.score_scale(K[b, 0, 0], q[0, 0], d))
+
+
+# ------------------------------------------------------------------ large pools: the streaming one-launch kernel
+@pytest.mark.parametrize("N,budget,lam", [(257, 40, 0.5), (300, 128, 0.0), (1000, 64, 0.5), (1000, 100, 1.5), (2050, 128, 1.0)])
+def test_large_pool_stream_kernel(N, budget, lam):
+    """bf16, d = 128, N > 256: K streams through a ring, scores stay on chip, pool rows of V only. Ragged
+    candidate counts put the end of an event inside a ring stage, at its edge, and below the budget."""
+    ev = synth.make_c3(seed=N, B=4, L=1, H=2, N=N, budget=budget)
+    before = akv.launch_count()
+    g = run_fused(ev, lam=lam)
+    assert akv.launch_count() == before + 1                                   # one launch for the whole event
+    check_all(ev, g, lam)
+    n_cand = [N, N - 63, 64 * (N // 64), budget - 3]
+    g = run_fused(ev, lam=lam, n_cand=n_cand)
+    check_all(ev, g, lam, n_cand=n_cand)
+
+
+def test_large_pool_stream_kernel_variants():
+    """Same kernel: no pruning (the pool outgrows the on-chip tile, the rest of V is read in place), the greedy
+    loop forced at lambda = 0, per-head budgets, irregular positions with the default reference position, every
+    row scored from scratch, and the bounded waits running out."""
+    ev = synth.make_c3(seed=71, B=2, L=2, H=2, N=900, budget=48)
+    base = run_fused(ev)
+    check_all(ev, base, ev.lam)
+    full = run_fused(ev, flags=akv.FLAG_NO_PRUNE)
+    for k in ("order", "idx", "K", "V", "pos"):
+        assert np.array_equal(base[k], full[k]), k
+    fast, loop = run_fused(ev, lam=0.0), run_fused(ev, lam=0.0, flags=akv.FLAG_FORCE_GREEDY)
+    assert np.array_equal(fast["order"], loop["order"]) and np.array_equal(fast["K"], loop["K"])
+    check_all(ev, fast, 0.0)
+    budgets = np.array([[48, 1], [17, 30]], dtype=np.int32)
+    check_all(ev, run_fused(ev, budgets=budgets), ev.lam, budgets=budgets)
+    fresh = run_fused(ev, flags=akv.FLAG_NO_CHAIN)
+    assert np.max(np.abs(fresh["scores"] - base["scores"])) < 2e-6
+    check_all(ev, fresh, ev.lam)
+    ev.pos[:] = np.sort(np.random.default_rng(72).choice(200_000, size=900, replace=False)).astype(np.int32)
+    g = run_fused(ev, p_ref=False)
+    check_all(ev, g, ev.lam, p_ref=False)
+    starved = run_fused(ev, flags=akv.FLAG_TEST_STARVE_WAIT)
+    assert np.all(starved["status"] == 3)
+    assert np.array_equal(starved["K"], ev.K) and np.array_equal(starved["V"], ev.V) and np.array_equal(starved["pos"], ev.pos)
+
+
+def test_large_pool_stream_kernel_paged():
+    c5 = synth.make_c5(seed=73, B=2, L=2, H=2, page=64, pages_per_seq=9, budget=100, rounds=1)   # N = 576
+    L, H, N, d, b = c5.L, c5.H, c5.N, c5.d, c5.budget
+    pool_K, pool_V = dev(c5.pool_K), dev(c5.pool_V)
+    table, pos, q = dev(c5.block_table), dev(c5.pos), dev(c5.qstat)
+    lay = akv.Layout.paged(pool_K, table)
+    hostK = synth.paged_gather_dense(c5.pool_K, c5.block_table)
+    hostV = synth.paged_gather_dense(c5.pool_V, c5.block_table)
+    sel = akv.alpha_compress_event(pool_K, pool_V, pos, q, b, akv.Options(lam=c5.lam), layout=lay, want_scores=True)
+    torch.cuda.synchronize()
+    idx, order, sc = sel.idx_sorted.cpu().numpy(), sel.pick_order.cpu().numpy(), sel.scores.cpu().numpy()
+    posn = pos.cpu().numpy()
+    for bb in range(c5.B):
+        pages = c5.block_table[bb].tolist()
+        for l in range(L):
+            for h in range(H):
+                Kn = akv.to_host_bits(pool_K[l, pages, h]).reshape(N, d)
+                Vn = akv.to_host_bits(pool_V[l, pages, h]).reshape(N, d)
+                chk.check_event(hostK[bb, l, h], hostV[bb, l, h], c5.pos[bb, l, h], c5.qstat[l, h], None, b, c5.lam,
+                                sc[bb, l, h], order[bb, l, h], idx[bb, l, h], Kn, Vn, posn[bb, l, h], log=[])
+
+
+def test_chained_and_fresh_scores_agree_on_the_tensor_memory_kernels():
+    for ev in (synth.make_c3(seed=81, B=2, L=2, H=2, N=192, budget=64), synth.make_c2(seed=82, B=1, L=2, H=2)):
+        a, b = run_fused(ev), run_fused(ev, flags=akv.FLAG_NO_CHAIN)
+        scale = np.abs(a["scores"]).max()
+        assert np.max(np.abs(a["scores"] - b["scores"])) < 1e-6 * max(scale, 1.0)
+        check_all(ev, b, ev.lam)
 
 
 def test_report_worst_score_error():

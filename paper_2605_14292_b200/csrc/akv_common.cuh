@@ -64,8 +64,17 @@ __device__ long long* g_phase_buf = nullptr;
 __device__ __forceinline__ void phase_stamp(int event, int k) {
     if (threadIdx.x == 0 && g_phase_buf) g_phase_buf[(long long)event * kPhaseSlots + k] = clock64();
 }
+// cycles spent in a repeated step, summed by thread 0: acc += clock64() at the end, -= at the start
+#define AKV_PHASE_ACC_DECL(name) long long name = 0
+#define AKV_PHASE_ACC_BEGIN(name) do { if (threadIdx.x == 0) name -= clock64(); } while (0)
+#define AKV_PHASE_ACC_END(name) do { if (threadIdx.x == 0) name += clock64(); } while (0)
+#define AKV_PHASE_ACC_STORE(event, k, name) do { if (threadIdx.x == 0 && g_phase_buf) g_phase_buf[(long long)(event) * kPhaseSlots + (k)] = name; } while (0)
 #else
 __device__ __forceinline__ void phase_stamp(int, int) {}
+#define AKV_PHASE_ACC_DECL(name)
+#define AKV_PHASE_ACC_BEGIN(name)
+#define AKV_PHASE_ACC_END(name)
+#define AKV_PHASE_ACC_STORE(event, k, name)
 #endif
 
 // ---- element access: 4 or 8 consecutive elements widened to fp32 -------------------------------

@@ -2,7 +2,7 @@
 // 256 rows that the other tensor-memory kernels hold): prefill compression, N = 4096 -> budget 128.
 // One CTA of nine warps per event.
 //
-//   1. K streams through a ring of four 64-row stages (cp.async.bulk + full/empty mbarriers, one
+//   1. K streams through a ring of eight 64-row stages (cp.async.bulk + full/empty mbarriers, one
 //      producer warp, eight scoring warps); every row is scored as it lands and only its score stays
 //      on chip. K is read from HBM exactly once.
 //   2. s_(b) by a radix-4 bisection over the score keys (all eight warps), then either the top-k
@@ -26,19 +26,21 @@ constexpr int kStWarps = 8;                        // scoring / selection warps
 constexpr int kStWork = kStWarps * 32;             // their threads
 constexpr int kStThreads = kStWork + 32;           // plus the producer warp
 constexpr int kStStageRows = 64;                   // K rows per ring stage
-constexpr int kStStages = 4;
+constexpr int kStMaxStages = 8;                    // ring depth: 8 stages (128 KB in flight per SM) when they fit, else 4
 constexpr unsigned kStStageBytes = kStStageRows * 256u;
-constexpr unsigned kStRingBytes = kStStages * kStStageBytes;
+constexpr unsigned kStStageChunk = 4u * kStStageBytes;  // kept rows of K and of V (128 each) staged on their way out
 constexpr int kStRoundRows = kStWarps * 4;         // rows scored per round (4 per warp)
 constexpr int kStCpl = 4;                          // candidates per thread: pools of up to 1024 rows on the tensor-core route
 constexpr int kStExtra = 256;                      // pool rows beyond the tile that the tensor-core route still takes
-constexpr int kStSpare = 16;                       // tile rows after the last pool row (window of a picked row; scratch row)
-constexpr uint32_t kStTmemCols = 128;              // 8 blocks of 128 pool rows x 16 columns
+constexpr int kStWin = 64;                         // pool rows whose cosine columns one product pass yields
+constexpr int kStSpare = kStWin;                   // tile rows after the last pool row (reach of a window; scratch row)
+constexpr uint32_t kStTmemCols = 512;              // 8 blocks of 128 pool rows x 64 columns
 
 struct StSmem {
     unsigned tile, pool, taken, xs, order, gain, idx, gtab, sect, slot, misc, total;
     unsigned tile_bytes, s, spos, rall, ptaken;  // offsets inside the tile region (valid until the V rows arrive)
     int cap_rows;                                // pool rows the operand tile holds
+    int stages;                                  // ring depth
 };
 // The tile region holds, in turn: the ring + scores + positions (scoring), the pool's V rows (selection), the
 // kept rows on their way out. The plain-dot route keeps its per-candidate arrays where the V rows would be.
@@ -52,13 +54,15 @@ __host__ __device__ inline StSmem plan_st_smem(int N, int budget, int smem_limit
     fixed += 3 * align16((unsigned)budget * 4);   // order, gain, idx
     fixed += 1024 + 256 + 256 + 256;              // gtab + phitab, sect, slot, misc
     fixed += 1024;                                // room to align the base to 1024 bytes
-    const unsigned need = kStRingBytes + 3 * align16(np * 4) + align16(np);  // ring, s, spos, rall, ptaken
+    const unsigned arrays = 3 * align16(np * 4) + align16(np);  // s, spos, rall, ptaken
     unsigned tile_bytes = (unsigned)smem_limit > fixed ? ((unsigned)smem_limit - fixed) / 2048u * 2048u : 0u;
     const unsigned max_tile = (1024u + kStSpare) * 256u;
     if (tile_bytes > max_tile) tile_bytes = max_tile;
     // whole blocks of 128 rows (a block's product reads all 128 of its rows), as long as the scoring phase still fits
-    if (tile_bytes / 32768u * 32768u >= need) tile_bytes = tile_bytes / 32768u * 32768u;
-    p.cap_rows = tile_bytes >= need ? (int)(tile_bytes / 256u) - kStSpare : 0;  // 0: the shape does not fit
+    if (tile_bytes / 32768u * 32768u >= 4u * kStStageBytes + arrays) tile_bytes = tile_bytes / 32768u * 32768u;
+    p.stages = tile_bytes >= (unsigned)kStMaxStages * kStStageBytes + arrays ? kStMaxStages : 4;
+    const unsigned ring = (unsigned)p.stages * kStStageBytes;
+    p.cap_rows = tile_bytes >= ring + arrays ? (int)(tile_bytes / 256u) - kStSpare : 0;  // 0: the shape does not fit
     p.tile_bytes = tile_bytes;
     unsigned o = 0;
     p.tile = o;   o += tile_bytes;
@@ -73,7 +77,7 @@ __host__ __device__ inline StSmem plan_st_smem(int N, int budget, int smem_limit
     p.slot = o;   o += 256;    // 2 x 8 arg-max keys of 8 bytes, 2 x 8 norms
     p.misc = o;   o += 256;    // mbarriers (full, empty, product), tensor-memory base, counters
     p.total = o + 1024;
-    p.s = kStRingBytes;
+    p.s = ring;
     p.spos = p.s + align16(np * 4);
     p.rall = p.spos + align16(np * 4);
     p.ptaken = p.rall + align16(np * 4);
@@ -121,11 +125,12 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     float2* sect = reinterpret_cast<float2*>(smem + sp.sect);
     unsigned long long* slot = reinterpret_cast<unsigned long long*>(smem + sp.slot);  // [2][8] keys
     float* slot_r = reinterpret_cast<float*>(smem + sp.slot + 128);                    // [2][8] norms of the warps' best
-    const uint32_t bar_full = smem_u32(smem + sp.misc);  // 4 barriers
-    const uint32_t bar_empty = bar_full + 32;            // 4 barriers
-    const uint32_t barM = bar_full + 64;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 72);
-    int* cnt = reinterpret_cast<int*>(smem + sp.misc + 80);  // [0] a wait ran out, [1] newest position
+    const uint32_t bar_full = smem_u32(smem + sp.misc);  // up to 8 barriers
+    const uint32_t bar_empty = bar_full + 64;            // up to 8 barriers
+    const uint32_t barM = bar_full + 128;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 136);
+    int* cnt = reinterpret_cast<int*>(smem + sp.misc + 144);  // [0] a wait ran out, [1] newest position
+    const int nst = sp.stages;
     const uint32_t tile_u32 = smem_u32(tile);
     const int cap = sp.cap_rows;
     const uint32_t half_bytes = (uint32_t)(cap + kStSpare) * 128u;
@@ -146,11 +151,10 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     phase_stamp(id.e, 0);  // phases: 0 start, 1 tables + positions, 2 K scored, 3 s_(b), 4 pool / top-k, 5 V rows + norms, 6 picks, 7 outputs, 8 end
     // ---- set-up: barriers, tables, positions on chip --------------------------------------------------------
     if (tid == 0) {
-        for (int i = 0; i < kStStages; ++i) {
+        for (int i = 0; i < nst; ++i) {
             mbar_init(bar_full + 8 * i, 1);
             mbar_init(bar_empty + 8 * i, kStWarps);
         }
-        mbar_init(barM, 1);
         mbar_init_fence();
         cnt[0] = 0;
         cnt[1] = INT_MIN;
@@ -179,8 +183,8 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     if (!worker) {
         if (lane == 0) {
             for (int st = 0; st < stages; ++st) {
-                const int sl = st % kStStages;
-                if (st >= kStStages && !mbar_wait_bounded(bar_empty + 8 * sl, (uint32_t)((st / kStStages - 1) & 1), a.wait_polls)) {
+                const int sl = st % nst;
+                if (st >= nst && !mbar_wait_bounded(bar_empty + 8 * sl, (uint32_t)((st / nst - 1) & 1), a.wait_polls)) {
                     atomicExch(&cnt[0], 1);
                     break;
                 }
@@ -200,40 +204,54 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
         }
     } else {
         const int grp = lane >> 3, f0 = (lane & 7) * 8;
-        // spacing of rows one round (32 slots) apart at the newest end: what a cache filled token by token has everywhere
-        const long long D = n > kStRoundRows ? (long long)spos[n - 1] - (long long)spos[n - 1 - kStRoundRows] : 0;
-        ChainScore cs;
-        cs.set_step(D, phitab + f0, sect);
+        // A lane group scores two rows of every stage, 32 slots apart, as two independent chains (the second
+        // hides the first one's latencies); each chain steps by one stage = 64 slots. D: the spacing of rows 64
+        // slots apart at the newest end, which a cache filled token by token has everywhere.
+        const long long D = n > kStStageRows ? (long long)spos[n - 1] - (long long)spos[n - 1 - kStStageRows] : 0;
+        const int D32 = (int)D;
+        const bool d_fits = (long long)D32 == D;
+        ChainScore ca, cb;  // cb uses ca's S
+        ca.set_step(D, phitab + f0, sect);
         for (int st = 0; st < stages; ++st) {
-            const int sl = st % kStStages;
-            if (!mbar_wait_bounded(bar_full + 8 * sl, (uint32_t)((st / kStStages) & 1), a.wait_polls)) {
+            const int sl = st % nst;
+            if (!mbar_wait_bounded(bar_full + 8 * sl, (uint32_t)((st / nst) & 1), a.wait_polls)) {
                 atomicExch(&cnt[0], 1);
                 break;
             }
-#pragma unroll 1
-            for (int rr = 0; rr < kStStageRows / kStRoundRows; ++rr) {
-                const int round = st * (kStStageRows / kStRoundRows) + rr;
-                const int j = round * kStRoundRows + 4 * warp + grp;
-                const bool live = j < n;
-                bool fresh = (round & (kChainRounds - 1)) == 0 || a.no_chain;
-                if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - kStRoundRows] == D);
-                if (fresh) {
-                    if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);
-                } else {
-                    cs.advance();
-                }
-                float acc = 0.f;
-                if (live) {
-                    const unsigned char* krow = tile + sl * kStStageBytes + (j - st * kStStageRows) * 256 + (lane & 7) * 16;
-                    acc = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
-                }
+            const int ja = st * kStStageRows + 4 * warp + grp, jb = ja + kStRoundRows;
+            const bool la = ja < n, lb = jb < n;
+            const int pa = la ? spos[ja] : 0, pb = lb ? spos[jb] : 0;
+            bool fresh = (st & (kChainRounds - 1)) == 0 || a.no_chain || !d_fits;
+            if (!fresh)
+                fresh = !__all_sync(0xFFFFFFFFu, (!la || pa - spos[ja - kStStageRows] == D32) && (!lb || pb - spos[jb - kStStageRows] == D32));
+            if (fresh) {
+                if (la) ca.anchor(pref - (long long)pa, gtab + f0, phitab + f0, sect);
+                if (lb) cb.anchor(pref - (long long)pb, gtab + f0, phitab + f0, sect);
+            } else {
+                ca.advance();
+                cb.advance_by(ca);
+            }
+            float acca = 0.f, accb = 0.f;
+            const unsigned char* krow = tile + sl * kStStageBytes + (4 * warp + grp) * 256 + (lane & 7) * 16;
+            if (la) acca = ca.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
+            if (lb) accb = cb.dot(*reinterpret_cast<const uint4*>(krow + kStRoundRows * 256), *reinterpret_cast<const uint4*>(krow + kStRoundRows * 256 + 128));
 #pragma unroll
-                for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-                if (live && (lane & 7) == 0) {
-                    if (a.scores) a.scores[(long long)id.e * N + j] = acc;
-                    const bool fin = isfinite(acc);
+            for (int off = 4; off > 0; off >>= 1) {
+                acca += __shfl_xor_sync(0xFFFFFFFFu, acca, off);
+                accb += __shfl_xor_sync(0xFFFFFFFFu, accb, off);
+            }
+            if ((lane & 7) == 0) {
+                if (la) {
+                    if (a.scores) a.scores[(long long)id.e * N + ja] = acca;
+                    const bool fin = isfinite(acca);
                     bad |= !fin;
-                    s[j] = fin ? acc : -INFINITY;
+                    s[ja] = fin ? acca : -INFINITY;
+                }
+                if (lb) {
+                    if (a.scores) a.scores[(long long)id.e * N + jb] = accb;
+                    const bool fin = isfinite(accb);
+                    bad |= !fin;
+                    s[jb] = fin ? accb : -INFINITY;
                 }
             }
             __syncwarp();
@@ -245,7 +263,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
         // a wait ran out: report it, give copies that may still be in flight a bounded chance to land, leave
         if (tid == 0) {
             if (a.status) a.status[id.e] = 3;
-            for (int sl = 0; sl < kStStages; ++sl) {
+            for (int sl = 0; sl < nst; ++sl) {
                 mbar_wait_bounded(bar_full + 8 * sl, 0, a.wait_polls);
                 mbar_wait_bounded(bar_full + 8 * sl, 1, a.wait_polls);
             }
@@ -262,18 +280,36 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     // ---- s_(b): the picks-th largest score key, two bits per round ---------------------------------------------
     uint32_t kb = 0u;
     if (picks > 0) {
+        // up to 16 keys per thread stay in registers (N <= 4096); longer events read theirs from shared memory
+        constexpr int kRegKeys = 16;
+        const bool in_regs = n <= kRegKeys * kStWork;
+        uint32_t kreg[kRegKeys];
+#pragma unroll
+        for (int i = 0; i < kRegKeys; ++i) {
+            const int j = tid + i * kStWork;
+            kreg[i] = (in_regs && j < n) ? orderable(s[j]) : 0u;
+        }
         for (int lo = 30; lo >= 0; lo -= 2) {
             const uint32_t v1 = kb | (1u << lo), v2 = kb | (2u << lo), v3 = kb | (3u << lo);
+            // the three counts of a warp (at most 512 each when the keys sit in registers) travel in one word
+            uint32_t c = 0u;
             int c1 = 0, c2 = 0, c3 = 0;
-            for (int j = tid; j < n; j += kStWork) {
-                const uint32_t k = orderable(s[j]);
-                c1 += k >= v1;
-                c2 += k >= v2;
-                c3 += k >= v3;
+            if (in_regs) {
+#pragma unroll
+                for (int i = 0; i < kRegKeys; ++i) c += (kreg[i] >= v1) + ((kreg[i] >= v2) << 10) + ((kreg[i] >= v3) << 20);
+                c = __reduce_add_sync(0xFFFFFFFFu, c);
+                c1 = c & 1023; c2 = (c >> 10) & 1023; c3 = c >> 20;
+            } else {
+                for (int j = tid; j < n; j += kStWork) {
+                    const uint32_t k = orderable(s[j]);
+                    c1 += k >= v1;
+                    c2 += k >= v2;
+                    c3 += k >= v3;
+                }
+                c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+                c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+                c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
             }
-            c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
-            c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
-            c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
             int (*rp)[3] = radix_part[(lo >> 1) & 1];  // per-warp partial counts, double-buffered by round
             if (lane == 0) { rp[warp][0] = c1; rp[warp][1] = c2; rp[warp][2] = c3; }
             work_barrier();
@@ -365,20 +401,57 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
             // is lane r of tensor memory, and a warp reads the lanes of its own quarter
             const int quarter = warp & 3, blk0 = warp >> 2;
             const int resident = min(P, cap), extras = P - resident;
+            // The pool goes into the tile by descending score (equal scores by slot): picks then come roughly in
+            // tile order, and one product pass, which yields the cosine columns of the 64 tile rows from the picked
+            // one on, serves the picks that follow until one falls outside that window.
+            {
+                unsigned long long* skey = reinterpret_cast<unsigned long long*>(spos);  // positions and the plain-dot arrays are dead
+                unsigned short* sorted = reinterpret_cast<unsigned short*>(xs);
+                for (int rho = tid; rho < P; rho += kStWork)
+                    skey[rho] = ((unsigned long long)orderable(s[pool[rho]]) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)rho);
+                work_barrier();
+                unsigned long long mine[kStCpl + 1];
+                int rank[kStCpl + 1];
+#pragma unroll
+                for (int k = 0; k <= kStCpl; ++k) {
+                    const int rho = tid + k * kStWork;
+                    mine[k] = rho < P ? skey[rho] : ~0ull;
+                    rank[k] = 0;
+                }
+                for (int o = 0; o < P; ++o) {
+                    const unsigned long long ko = skey[o];
+#pragma unroll
+                    for (int k = 0; k <= kStCpl; ++k) rank[k] += ko > mine[k];
+                }
+#pragma unroll
+                for (int k = 0; k <= kStCpl; ++k) {
+                    const int rho = tid + k * kStWork;
+                    if (rho < P) sorted[rank[k]] = pool[rho];
+                }
+                work_barrier();
+                for (int rho = tid; rho < P; rho += kStWork) pool[rho] = sorted[rho];
+                work_barrier();
+            }
             float sv[kStCpl], lr[kStCpl], rr[kStCpl], M[kStCpl];
+            uint32_t klow[kStCpl];  // low key word: 0xFFFF - slot (ties go to the lower slot), then the pool row
             uint32_t alive = 0u;
 #pragma unroll
             for (int k = 0; k < kStCpl; ++k) {
                 const int rho = 128 * (2 * k + blk0) + 32 * quarter + lane;
-                sv[k] = 0.f; lr[k] = 0.f; rr[k] = 0.f; M[k] = 0.f;
+                sv[k] = 0.f; lr[k] = 0.f; rr[k] = 0.f; M[k] = 0.f; klow[k] = 0u;
                 if (rho < resident) {
-                    sv[k] = s[pool[rho]];
+                    const int j = pool[rho];
+                    sv[k] = s[j];
+                    klow[k] = ((0xFFFFu - (uint32_t)j) << 16) | (uint32_t)rho;
                     alive |= 1u << k;
                 }
             }
+            uint32_t xklow = 0u;
             if (tid < extras) {
-                xs[tid] = s[pool[resident + tid]];
+                const int j = pool[resident + tid];
+                xs[tid] = s[j];
                 xM[tid] = 0.f;
+                xklow = ((0xFFFFu - (uint32_t)j) << 16) | (uint32_t)(resident + tid);
             }
             bool xalive = tid < extras;
             if (warp == 0) tmem_alloc(smem_u32(tmem_holder), kStTmemCols);
@@ -408,37 +481,55 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
                     lr[k] = a.lam * rr[k];
                 }
             }
+            // a row beyond the tile stays in its thread's registers for the whole loop (256 bytes)
+            uint4 own[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) own[c] = make_uint4(0u, 0u, 0u, 0u);
             if (xalive) {
                 const __nv_bfloat16* vrow = Vg + rowoff(pool[resident + tid]);
                 float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(vrow + c * 8);
-                    dot8_bf16(v, v, acc);
+                    own[c] = *reinterpret_cast<const uint4*>(vrow + c * 8);
+                    dot8_bf16(own[c], own[c], acc);
                 }
                 xr[tid] = 1.f / (sqrtf(acc.x + acc.y) + a.eps);
                 xlr[tid] = a.lam * xr[tid];
             }
-            phase_stamp(id.e, 5);
             const int nblk = (resident + 127) >> 7;
-            const uint32_t idesc = umma_idesc_bf16(128, 16);
+            // window: 128 tile rows when the pool has at most four blocks (4 x 128 columns of tensor memory), else 64;
+            // it starts a little before the picked row, because a candidate that an earlier pick's penalty held back
+            // is picked later, behind the front of the sequence
+            const int win = nblk <= 4 ? 2 * kStWin : kStWin, back = nblk <= 4 ? 40 : 24;
+            const uint32_t idesc = umma_idesc_bf16(128, win);
+            int cbase = -1;  // first tile row of the window whose columns tensor memory holds (-1: none)
+            // block w's product is issued by lane 0 of warp w (blocks are independent: own rows, own columns), each
+            // with its own commit; the barrier completes when all nblk of them have arrived
+            if (tid == 0) {
+                mbar_init(barM, (uint32_t)nblk);
+                mbar_init_fence();
+            }
+            work_barrier();
             int timeout = 0;
             uint32_t mround = 0;
+            AKV_PHASE_ACC_DECL(cyc_argmax);
+            AKV_PHASE_ACC_DECL(cyc_product);
+            AKV_PHASE_ACC_DECL(cyc_update);
+            phase_stamp(id.e, 5);
             for (int t = 0; t < picks; ++t) {
+                AKV_PHASE_ACC_BEGIN(cyc_argmax);
                 // Eq. 2 for the candidates still competing, Eq. 3's arg-max (ties to the lower pool row = lower slot)
                 unsigned long long best = 0ull;
                 float best_r = 0.f;
 #pragma unroll
                 for (int k = 0; k < kStCpl; ++k) {
                     if (alive & (1u << k)) {
-                        const int rho = 128 * (2 * k + blk0) + 32 * quarter + lane;
-                        const unsigned long long key = ((unsigned long long)orderable(fmaf(-lr[k], M[k], sv[k])) << 32) |
-                                                       (unsigned long long)(0xFFFFFFFFu - (uint32_t)rho);
+                        const unsigned long long key = ((unsigned long long)orderable(fmaf(-lr[k], M[k], sv[k])) << 32) | klow[k];
                         if (key > best) { best = key; best_r = rr[k]; }
                     }
                 }
                 if (xalive) {
-                    const unsigned long long key = ((unsigned long long)orderable(fmaf(-xlr[tid], xM[tid], xs[tid])) << 32) |
-                                                   (unsigned long long)(0xFFFFFFFFu - (uint32_t)(resident + tid));
+                    const unsigned long long key = ((unsigned long long)orderable(fmaf(-xlr[tid], xM[tid], xs[tid])) << 32) | xklow;
                     if (key > best) { best = key; best_r = xr[tid]; }
                 }
                 if (timeout) best = ~0ull;
@@ -448,47 +539,56 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
                     timeout = 1;
                     break;
                 }
-                const int irho = key_row(top);
+                AKV_PHASE_ACC_END(cyc_argmax);
+                const int irho = (int)((uint32_t)top & 0xFFFFu);
                 if (tid == 0) order[t] = pool[irho];
 #pragma unroll
                 for (int k = 0; k < kStCpl; ++k)
                     if (128 * (2 * k + blk0) + 32 * quarter + lane == irho) alive &= ~(1u << k);
                 if (resident + tid == irho) xalive = false;
                 if (t + 1 == picks) break;
-                // cosines of the picked row against the pool: per block of 128 rows, block x (16 tile rows around the picked one)^T
-                int base = irho & ~7;
-                if (irho >= resident) {
-                    // the picked row lies beyond the tile: it becomes the scratch row after the last pool row
-                    base = cap;
-                    if (tid < 16) cp_async16(tile_u32 + tile_chunk(cap, tid, half_bytes), Vg + rowoff(pool[irho]) + tid * 8);
-                    cp_async_wait_all();
-                    fence_proxy_async();
-                    work_barrier();
-                }
-                const int col = irho >= resident ? 0 : irho - base;
-                if (tid == 0) {
-                    tc_fence_after();
-                    for (int blk = 0; blk < nblk; ++blk) {
+                // cosines of the picked row against the pool: already in tensor memory when the row lies in the current
+                // window; else one product per block of 128 rows, block x (the 64 tile rows from the picked one on)^T
+                const bool hit = irho < resident && cbase >= 0 && irho >= cbase && irho < cbase + win;
+                AKV_PHASE_ACC_BEGIN(cyc_product);
+                if (!hit) {
+                    cbase = max(irho - back, 0) & ~7;
+                    if (irho >= resident) {
+                        // the picked row lies beyond the tile: it becomes the scratch row after the last pool row
+                        cbase = cap;
+                        if (tid < 16) cp_async16(tile_u32 + tile_chunk(cap, tid, half_bytes), Vg + rowoff(pool[irho]) + tid * 8);
+                        cp_async_wait_all();
+                        fence_proxy_async();
+                        work_barrier();
+                    }
+                    if (lane == 0 && warp < nblk) {
+                        tc_fence_after();
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
-                            umma_bf16(tbase + (uint32_t)(16 * blk), umma_desc_sw128(tile_u32 + (uint32_t)blk * 16384u + koff),
-                                      umma_desc_sw128(tile_u32 + (uint32_t)base * 128u + koff), idesc, kk > 0 ? 1u : 0u);
+                            umma_bf16(tbase + (uint32_t)(win * warp), umma_desc_sw128(tile_u32 + (uint32_t)warp * 16384u + koff),
+                                      umma_desc_sw128(tile_u32 + (uint32_t)cbase * 128u + koff), idesc, kk > 0 ? 1u : 0u);
                         }
+                        umma_commit(barM);
                     }
-                    umma_commit(barM);
                 }
+                const int col = irho >= resident ? 0 : irho - cbase;
                 // rows beyond the tile: plain dot products, both rows read in place, while the tensor core works
                 if (xalive) {
-                    const __nv_bfloat16* vrow = Vg + rowoff(pool[resident + tid]);
-                    const __nv_bfloat16* vpick = Vg + rowoff(pool[irho]);
+                    const int prow = irho >= resident ? cap : irho;  // the picked row sits in the tile (as the scratch row if need be)
                     float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
                     for (int c = 0; c < 16; ++c)
-                        dot8_bf16(*reinterpret_cast<const uint4*>(vrow + c * 8), *reinterpret_cast<const uint4*>(vpick + c * 8), acc);
+                        dot8_bf16(own[c], *reinterpret_cast<const uint4*>(tile + tile_chunk(prow, c, half_bytes)), acc);
                     xM[tid] = fmaxf(xM[tid], ri * (acc.x + acc.y));
                 }
-                if (!mbar_wait_bounded(barM, mround & 1u, a.wait_polls)) timeout = 1;  // offered to everyone at the next exchange
-                ++mround;
+                if (!hit) {
+                    if (!mbar_wait_bounded(barM, mround & 1u, a.wait_polls)) timeout = 1;  // offered to everyone at the next exchange
+                    ++mround;
+                    if (irho >= resident) cbase = -1;  // the scratch row's window serves this pick only
+                }
+                AKV_PHASE_ACC_END(cyc_product);
+                AKV_PHASE_ACC_BEGIN(cyc_update);
                 tc_fence_after();
                 {
                     // tcgen05.ld is a warp-wide instruction: every lane issues it, for every block the pool has
@@ -497,7 +597,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
 #pragma unroll
                     for (int k = 0; k < kStCpl; ++k)
                         dv[k] = (2 * k + blk0 < nblk)
-                                    ? tmem_ld1(tbase + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(16 * (2 * k + blk0) + col))
+                                    ? tmem_ld1(tbase + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(win * (2 * k + blk0) + col))
                                     : 0.f;
                     tmem_ld_wait();
 #pragma unroll
@@ -505,7 +605,11 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
                         if (alive & (1u << k)) M[k] = fmaxf(M[k], ri * dv[k]);
                 }
                 tc_fence_before();
+                AKV_PHASE_ACC_END(cyc_update);
             }
+            AKV_PHASE_ACC_STORE(id.e, 10, cyc_argmax);
+            AKV_PHASE_ACC_STORE(id.e, 11, cyc_product);
+            AKV_PHASE_ACC_STORE(id.e, 12, cyc_update);
             tc_fence_before();
             work_barrier();
             if (warp == 0) tmem_dealloc(tbase, kStTmemCols);
@@ -589,16 +693,9 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
 
     phase_stamp(id.e, 6);
     // ---- sort(S) and outputs -------------------------------------------------------------------------
-    if (warp == 0) {
-        int off = 0;
-        for (int base = 0; base < n; base += 32) {
-            const int j = base + lane;
-            const bool f = j < n && taken[j];
-            const unsigned mask = __ballot_sync(0xFFFFFFFFu, f);
-            if (f) idx[off + __popc(mask & ((1u << lane) - 1u))] = j;
-            off += __popc(mask);
-        }
-        for (int t = off + lane; t < a.budget; t += 32) idx[t] = -1;
+    {
+        const int kept = ordered_scan([&](int j) { return taken[j] != 0; }, [&](int j, int pos) { idx[pos] = j; });
+        for (int t = kept + tid; t < a.budget; t += kStWork) idx[t] = -1;
     }
     work_barrier();
     const long long ob = (long long)id.e * a.budget;
@@ -617,7 +714,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     // (a chunk's destinations [c0, c1) can only be sources of the same or of later chunks: idx is ascending
     // and idx[t] >= t; later chunks' sources lie at or beyond their own destinations)
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
-    const int chunk = (int)(kStRingBytes / 512u);  // rows of K and V together that the ring region holds
+    const int chunk = (int)(kStStageChunk / 512u);  // rows of K and of V staged per round
     for (int c0 = 0; c0 < picks; c0 += chunk) {
         const int cn = min(chunk, picks - c0);
         work_barrier();

@@ -59,6 +59,15 @@ struct ChainScore {
             Gx[p] = nx; Gy[p] = ny;
         }
     }
+    // the same turn, taken from another state's S (two rows of a lane group chained side by side share one S)
+    __device__ __forceinline__ void advance_by(const ChainScore& o) {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float2 nx = __ffma2_rn(Gy[p], o.nSy[p], __fmul2_rn(Gx[p], o.Sx[p]));
+            const float2 ny = __ffma2_rn(Gy[p], o.Sx[p], __fmul2_rn(Gx[p], o.Sy[p]));
+            Gx[p] = nx; Gy[p] = ny;
+        }
+    }
     // the lane's partial sum of Re(G conj(k)) over its 8 frequencies
     __device__ __forceinline__ float dot(const uint4& wr, const uint4& wi) const {
         const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};

@@ -71,6 +71,9 @@ def main():
         d = (st[ok, k + 1] - st[ok, k]).astype(np.float64)
         if d.size:
             print(f"  {name:32s} {np.median(d):10.0f} {d.mean():10.0f}")
+    if kernel == "event_stream_kernel" and np.any(st[:, 10] > 0):
+        for k, name in ((10, "  of picks: arg-max + exchange"), (11, "  of picks: products (misses)"), (12, "  of picks: tensor-memory read")):
+            print(f"  {name:32s} {np.median(st[:, k]):10.0f} {st[:, k].mean():10.0f}")
     life = (st[:, len(names)] - st[:, 0]).astype(np.float64)
     life = life[(st[:, len(names)] > 0) & (st[:, 0] > 0)]
     print(f"  {'CTA lifetime':32s} {np.median(life):10.0f} {life.mean():10.0f}")

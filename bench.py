@@ -43,8 +43,8 @@ WORKLOADS = {
           "d=128, bf16, lambda=0.5",
 }
 # kernel(s) one call of the fused entry point launches for each workload
-KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_tc_kernel<fused>", "C3": "event_tri_kernel<fused>",
-           "C4": "event_stream_kernel", "C5": "event_tc_kernel<fused>"}
+KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_pool_kernel<fused>", "C3": "event_tri_kernel<fused>",
+           "C4": "event_stream_kernel", "C5": "event_pool_kernel<fused>"}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per step from the ncu captures summarised under profiles/,
 # keyed by workload, each with the source revision of csrc/ it was taken at (see kernel_revision()); a

@@ -18,7 +18,7 @@
 //      dot products from global memory; a pool that exceeds even that takes a plain-dot loop.
 //   5. Kept K and V rows are staged on chip and written to slots 0..b-1 of the same buffers.
 #pragma once
-#include "akv_event_tc.cuh"
+#include "akv_event_pool.cuh"
 
 namespace akv {
 
@@ -32,6 +32,7 @@ constexpr unsigned kStStageChunk = 4u * kStStageBytes;  // kept rows of K and of
 constexpr int kStRoundRows = kStWarps * 4;         // rows scored per round (4 per warp)
 constexpr int kStCpl = 4;                          // candidates per thread: pools of up to 1024 rows on the tensor-core route
 constexpr int kStExtra = 256;                      // pool rows beyond the tile that the tensor-core route still takes
+constexpr int kStActive = 248;                     // rows of the active set whose cosine matrix goes to shared memory as a triangle
 constexpr int kStWin = 64;                         // pool rows whose cosine columns one product pass yields
 constexpr int kStSpare = kStWin;                   // tile rows after the last pool row (reach of a window; scratch row)
 constexpr uint32_t kStTmemCols = 512;              // 8 blocks of 128 pool rows x 64 columns
@@ -395,8 +396,136 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
         P = ordered_scan([&](int j) { return !(s[j] < thr); }, [&](int j, int pos) { pool[pos] = (unsigned short)j; });
 
         phase_stamp(id.e, 4);
-        if (P <= cap + kStExtra && picks > 1) {
-            // ======== tensor-core route ==========================================================================
+        // ======== active-set route ===============================================================================
+        // The picks hardly ever reach beyond the best-scored few dozen rows past the budget. So: the cosine matrix
+        // of the pool's kStActive best-scored rows only (one tcgen05 product per block of 128 rows, lower triangle
+        // to shared memory), and Algorithm 1 as a one-warp loop over that triangle. Every candidate left out
+        // scores at most `bound` and its Eq. 2 value never exceeds its score, so the loop is exact as long as the
+        // winning value stays above the bound; if it ever does not, the event is redone by the routes below.
+        bool done = false;
+        if (picks > 1 && cap >= 256) {
+            // the (kStActive + 1)-th largest key of the pool (0: the pool is no larger than the active set)
+            uint32_t bound = 0u;
+            if (P > kStActive) {
+                uint32_t pk[kStCpl + 1];
+#pragma unroll
+                for (int k = 0; k <= kStCpl; ++k) {
+                    const int rho = tid + k * kStWork;
+                    pk[k] = rho < P ? orderable(s[pool[rho]]) : 0u;
+                }
+                const bool in_regs = P <= (kStCpl + 1) * kStWork;
+                for (int lo = 30; lo >= 0; lo -= 2) {
+                    const uint32_t v1 = bound | (1u << lo), v2 = bound | (2u << lo), v3 = bound | (3u << lo);
+                    int c1 = 0, c2 = 0, c3 = 0;
+                    if (in_regs) {
+#pragma unroll
+                        for (int k = 0; k <= kStCpl; ++k) { c1 += pk[k] >= v1; c2 += pk[k] >= v2; c3 += pk[k] >= v3; }
+                    } else {
+                        for (int rho = tid; rho < P; rho += kStWork) {
+                            const uint32_t k = orderable(s[pool[rho]]);
+                            c1 += k >= v1; c2 += k >= v2; c3 += k >= v3;
+                        }
+                    }
+                    c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+                    c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+                    c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+                    int (*rp)[3] = radix_part[(lo >> 1) & 1];
+                    if (lane == 0) { rp[warp][0] = c1; rp[warp][1] = c2; rp[warp][2] = c3; }
+                    work_barrier();
+                    int t1 = 0, t2 = 0, t3 = 0;
+#pragma unroll
+                    for (int w = 0; w < kStWarps; ++w) { t1 += rp[w][0]; t2 += rp[w][1]; t3 += rp[w][2]; }
+                    bound = t3 > kStActive ? v3 : (t2 > kStActive ? v2 : (t1 > kStActive ? v1 : bound));
+                }
+            }
+            // the active rows, in slot order (ties in the loop then go to the lower row = the lower slot)
+            unsigned short* act = reinterpret_cast<unsigned short*>(xs);  // 256 entries
+            float* ar = xs + 128;                                          // their reciprocal norms: 256 floats
+            const int R = ordered_scan([&](int j) { return !(s[j] < thr) && orderable(s[j]) > bound; },
+                                       [&](int j, int pos) { act[pos] = (unsigned short)j; });
+            if (warp == 0) tmem_alloc(smem_u32(tmem_holder), kStTmemCols);
+            for (int x = tid; x < R * 16; x += kStWork) {
+                const int rho = x >> 4, c = x & 15;
+                cp_async16(tile_u32 + tile_chunk(rho, c, half_bytes), Vg + rowoff(act[rho]) + c * 8);
+            }
+            if (tid == 0) {
+                mbar_init(barM, 1);
+                mbar_init_fence();
+            }
+            cp_async_wait_all();
+            fence_proxy_async();
+            tc_fence_before();
+            work_barrier();
+            tc_fence_after();
+            const uint32_t tbase = *tmem_holder;
+            const int nblk = (R + 127) >> 7, ncol = (R + 15) & ~15;
+            if (tid == 0) {
+                const uint32_t idesc = umma_idesc_bf16(128, ncol);
+                for (int blk = 0; blk < nblk; ++blk) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t koff = (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
+                        umma_bf16(tbase + (uint32_t)(256 * blk), umma_desc_sw128(tile_u32 + (uint32_t)blk * 16384u + koff),
+                                  umma_desc_sw128(tile_u32 + koff), idesc, kk > 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(barM);
+            }
+            int timeout = !mbar_wait_bounded(barM, 0, a.wait_polls);
+            tc_fence_after();
+            // every thread has seen the product complete (it has read the whole tile) before the triangle lands on the tile
+            timeout = __reduce_or_sync(0xFFFFFFFFu, timeout);
+            if (lane == 0 && timeout) atomicExch(&cnt[0], 1);
+            work_barrier();
+            if (!cnt[0]) {
+                // lower triangle -> shared memory: warp w holds rows 128 (w / 4) + 32 (w % 4) + lane of the matrix
+                float* tri = reinterpret_cast<float*>(tile);
+                const int blk = warp >> 2, row = 128 * blk + 32 * (warp & 3) + lane;
+                if (128 * blk + 32 * (warp & 3) < R) {
+                    const uint32_t lanes = tbase + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(256 * blk);
+                    const int trow = tri_row(row), last_cb = (128 * blk + 32 * (warp & 3) + 31) >> 5;
+                    for (int cb = 0; cb <= last_cb; ++cb) {
+                        uint32_t v[32];
+                        tmem_ld32(lanes + (uint32_t)(32 * cb), v);
+                        tmem_ld_wait();
+                        if (row < R) {
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) {
+                                if (32 * cb + k <= row) tri[trow + 32 * cb + k] = __uint_as_float(v[k]);
+                                if (32 * cb + k == row) ar[row] = 1.f / (sqrtf(__uint_as_float(v[k])) + a.eps);  // the diagonal: squared norm
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            work_barrier();
+            if (warp == 0) tmem_dealloc(tbase, kStTmemCols);
+            if (cnt[0]) {
+                if (tid == 0 && a.status) a.status[id.e] = 3;
+                return;
+            }
+            phase_stamp(id.e, 5);
+            if (warp == 0) {
+                const bool ok = picks_bounded<8, true>(lane, R, picks, true, s, act, ar, a.lam, reinterpret_cast<const float*>(tile),
+                                                           reinterpret_cast<uint32_t*>(gain), order, bound);
+                if (lane == 0) cnt[2] = ok ? 1 : 0;
+            }
+            work_barrier();
+            done = cnt[2] != 0;
+            if (done) {
+                for (int t = tid; t < picks; t += kStWork) {
+                    const int j = act[order[t]];
+                    gain[t] = from_orderable(reinterpret_cast<uint32_t*>(gain)[t]);
+                    order[t] = j;
+                }
+            }
+            work_barrier();
+        }
+        if (done) {
+            // picks are in order[] / gain[]
+        } else if (P <= cap + kStExtra && picks > 1) {
+            // ======== tensor-core route: any pool that fits the tile (a few rows may stay outside) ================
             // thread (warp w, lane l) owns pool rows 128 (2 k + w / 4) + 32 (w % 4) + l, k < 4: row r of a block of 128
             // is lane r of tensor memory, and a warp reads the lanes of its own quarter
             const int quarter = warp & 3, blk0 = warp >> 2;

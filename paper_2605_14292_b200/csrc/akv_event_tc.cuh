@@ -25,7 +25,7 @@ constexpr int kTcThreads = 128;
 constexpr int kTcD = 128;        // head dimension of this path
 constexpr int kTcMaxN = 256;     // most candidates per event
 constexpr int kTcCols = 128;     // cosine-matrix columns kept in tensor memory per block of 128 rows
-constexpr int kWaitPolls = 1 << 22;
+constexpr int kWaitPolls = 1 << 20;  // most polls of a bounded wait (the time-bounded form usually stops by its clock first)
 
 struct TcSmem {
     unsigned tile, s, key, spos, byrank, rankof, taken, order, gain, idx, sect, slot, misc, total;
@@ -77,10 +77,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up after `polls` polls, or after kWaitNs of wall-clock time (a poll may itself
 // suspend the thread for a while, so a poll count alone can stand for minutes), instead of spinning for ever.
+// The first poll is inline; the loop behind it is one out-of-line routine, so that a wait costs the
+// kernels a handful of instructions where the data is already there.
 constexpr unsigned long long kWaitNs = 200ull * 1000ull * 1000ull;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int polls) {
+__device__ __noinline__ bool mbar_wait_loop(uint32_t bar, uint32_t parity, int polls) {
     unsigned long long t0 = 0ull;
-    for (int it = 0; it < polls; ++it) {
+    for (int it = 1; it < polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63) == 63) {
             unsigned long long now;
@@ -89,6 +91,18 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
             else if (now - t0 > kWaitNs) return false;
         }
     }
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int polls) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_loop(bar, parity, polls);
+}
+// The plain form: a poll count only (2^20 polls: seconds at most, whatever a poll costs), all inline. The small
+// event kernel uses it: its register allocation and schedule, and with them 7 % of its speed, depend on it.
+constexpr int kWaitPollsPlain = 1 << 20;
+__device__ __forceinline__ bool mbar_wait_polls(uint32_t bar, uint32_t parity, int polls) {
+    for (int it = 0; it < polls; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

@@ -181,7 +181,7 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
 template <bool FUSED>
-__global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
+__global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const DevLayout& lay = a.lay;
@@ -250,7 +250,11 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
         mbar_init(barL, 1);
         mbar_init_fence();
     }
-    if (FUSED && warp == 1) fill_sector_table(sect, lane);
+    if (FUSED && tid >= 32 && tid < 64) {
+        float sn, cs;
+        sincospif((float)(tid - 32) * 0.0625f, &sn, &cs);  // angle 2 pi h / 32
+        sect[tid - 32] = make_float2(cs, sn);
+    }
     if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), kTcCols);
     tc_fence_before();
     __syncthreads();
@@ -275,7 +279,14 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
         // shared memory (storage that the selection uses later)
         float2* gtab = reinterpret_cast<float2*>(smem + sp.bypool);
         unsigned long long* phitab = reinterpret_cast<unsigned long long*>(gtab + 64);
-        fill_statistic_tables(a.qstat + ((long long)id.l * lay.H + id.h) * kTcD, tab, tid, gtab, phitab);
+        if (tid < 64) {
+            const float* q = a.qstat + ((long long)id.l * lay.H + id.h) * kTcD;
+            const float inv = rsqrtf((float)kTcD);
+            const float qr = q[tid] * inv, qi = q[tid + 64] * inv;
+            const float2 c = tab.cw[tid];
+            gtab[tid] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+            phitab[tid] = tab.phi[tid];
+        }
         if (rotate) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) pmax = max(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, off));
@@ -325,11 +336,11 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
                 }
             }
         };
-        timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
+        timeout = !mbar_wait_polls(barK, 0, a.wait_polls);
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
             // first and third stretch share one copy of the loop (the kernel's code should stay small)
-            if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0, a.wait_polls);
+            if (pass && n_late > 0) timeout |= !mbar_wait_polls(barL, 0, a.wait_polls);
             score_rounds(pass ? kTriTileRows / 16 : 0, pass ? rounds : late_round);
             if (!pass) {
                 if (n_late > 0) {
@@ -353,8 +364,8 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
     timeout = __syncthreads_or(timeout);
     if (timeout) {
         if (tid == 0 && a.status) a.status[id.e] = 3;
-        mbar_wait_bounded(barK, 0, a.wait_polls);  // give copies still in flight another bounded chance to land
-        if (n_late > 0) mbar_wait_bounded(barL, 0, a.wait_polls);
+        mbar_wait_polls(barK, 0, a.wait_polls);  // give copies still in flight another bounded chance to land
+        if (n_late > 0) mbar_wait_polls(barL, 0, a.wait_polls);
         if (use_tc && warp == 0) tmem_dealloc(tbase, kTcCols);
         return;
     }
@@ -441,7 +452,7 @@ __global__ void __launch_bounds__(kTcThreads, 7) event_tri_kernel(const EventArg
             }
             umma_commit(barM);
         }
-        timeout = !mbar_wait_bounded(barM, 0, a.wait_polls);
+        timeout = !mbar_wait_polls(barM, 0, a.wait_polls);
         tc_fence_after();
     }
     timeout = __syncthreads_or(timeout);  // also: the product has read the whole tile before the triangle lands on it

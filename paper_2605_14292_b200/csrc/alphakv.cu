@@ -8,7 +8,7 @@
 #include <cstdio>
 #include <cstring>
 
-#include "akv_event_tri.cuh"
+#include "akv_event_pool.cuh"
 #include "akv_event_stream.cuh"
 #include "akv_select_pool.cuh"
 
@@ -311,15 +311,25 @@ static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t s
     return launched(FUSED ? "event_tc" : "select_tc");
 }
 
-// Single-warp greedy loop over a triangle of the pool's cosine matrix: the shapes whose pruned pool
-// normally stays within 128 rows.
+// Single-warp greedy loop over a triangle of the cosine matrix in shared memory. Small size: the shapes whose
+// pruned pool normally stays within 127 rows (N <= 128 or budget <= 64). Large size: budgets up to 128 with
+// N <= 256, over an active set of the pool's 152 best-scored rows.
 static bool tri_path_ok(const EventArgs& a) { return tc_path_ok(a) && (a.lay.N <= 128 || a.budget <= 64); }
-template <bool FUSED>
+static bool tri_big_ok(const EventArgs& a) { return tc_path_ok(a) && !tri_path_ok(a) && a.budget <= 128; }
+template <bool FUSED, bool BIG>
 static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
-    const TriSmem sp = plan_tri_smem(a.lay.N, a.budget);
+    const TriSmem sp = BIG ? plan_tri_smem(a.lay.N, a.budget, true) : plan_tri_smem(a.lay.N, a.budget);
     if ((int)sp.total > h->smem_optin) return fail(AKV_ERR_UNSUPPORTED, "budget %d needs too much shared memory", a.budget);
     akv_status_t s;
+    if (BIG) {
+        if ((s = set_smem(event_pool_kernel<FUSED, true>, sp.total)) != AKV_OK) return s;
+        CUDA_TRY(cudaFuncSetAttribute(event_pool_kernel<FUSED, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+        if (dry) return AKV_OK;
+        event_pool_kernel<FUSED, true><<<E, kTcThreads, sp.total, st>>>(a, h->tab);
+        return launched(FUSED ? "event_pool" : "select_pool_active");
+    }
     if ((s = set_smem(event_tri_kernel<FUSED>, sp.total)) != AKV_OK) return s;
     CUDA_TRY(cudaFuncSetAttribute(event_tri_kernel<FUSED>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                   (int)cudaSharedmemCarveoutMaxShared));
@@ -329,7 +339,8 @@ static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t s
 }
 
 static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
-    if (tri_path_ok(a) && a.V) return launch_tri<false>(h, a, st, dry);
+    if (tri_path_ok(a) && a.V) return launch_tri<false, false>(h, a, st, dry);
+    if (tri_big_ok(a) && a.V) return launch_tri<false, true>(h, a, st, dry);
     if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st, dry);
     return a.lay.dtype == AKV_BF16 ? launch_select_t<__nv_bfloat16>(h, a, st, dry) : launch_select_t<float>(h, a, st, dry);
 }
@@ -475,7 +486,7 @@ static akv_status_t kv_compact_impl(akv_handle_t* h, const akv_layout_t* lay, vo
 // Which kernels the fused call runs for a shape: the two tensor-memory kernels (bf16, d = 128, N <= 256,
 // per-head signatures), the resident kernel when an event's K and V tiles fit in shared memory, else
 // three launches with the scores in global memory.
-enum EventRoute { ROUTE_TRI, ROUTE_TC, ROUTE_STREAM, ROUTE_RESIDENT, ROUTE_THREE };
+enum EventRoute { ROUTE_TRI, ROUTE_TRI_BIG, ROUTE_TC, ROUTE_STREAM, ROUTE_RESIDENT, ROUTE_THREE };
 // shared memory the streaming kernel may plan with: what the device allows minus its static arrays
 static int stream_smem_limit(int smem_optin) { return smem_optin - 1024; }
 static bool stream_path_ok(const EventArgs& a, int smem_optin) {
@@ -485,6 +496,7 @@ static bool stream_path_ok(const EventArgs& a, int smem_optin) {
 }
 static EventRoute event_route(const EventArgs& a, int smem_optin) {
     if (tri_path_ok(a)) return ROUTE_TRI;
+    if (tri_big_ok(a)) return ROUTE_TRI_BIG;
     if (tc_path_ok(a)) return ROUTE_TC;
     if (stream_path_ok(a, smem_optin)) return ROUTE_STREAM;
     const int es = a.lay.dtype == AKV_BF16 ? 2 : 4;
@@ -557,7 +569,8 @@ static akv_status_t alpha_compress_event_impl(akv_handle_t* h, const akv_layout_
     a.scores = scores; a.n_kept = n_kept; a.status = status;
 
     const EventRoute route = event_route(a, h->smem_optin);
-    if (route == ROUTE_TRI) return launch_tri<true>(h, a, st);
+    if (route == ROUTE_TRI) return launch_tri<true, false>(h, a, st);
+    if (route == ROUTE_TRI_BIG) return launch_tri<true, true>(h, a, st);
     if (route == ROUTE_TC) return launch_tc<true>(h, a, st);
     if (route == ROUTE_STREAM) {
         const int limit = stream_smem_limit(h->smem_optin);

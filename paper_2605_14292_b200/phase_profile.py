@@ -39,7 +39,7 @@ def main():
     slots = int(lib.akv_debug_phase_slots())
     dev = torch.device("cuda")
     if args.config == "C2":
-        ev, kernel = synth.make_c2(B=args.batch or 1), "event_tc_kernel"
+        ev, kernel = synth.make_c2(B=args.batch or 1), "event_tri_kernel"
     elif args.config == "C3":
         ev, kernel = synth.make_c3(B=args.batch or 16), "event_tri_kernel"
     elif args.config == "C4":
@@ -50,7 +50,7 @@ def main():
         V = synth.paged_gather_dense(c5.pool_V, c5.block_table)
         ev = synth.EventBatch("C5-round0", synth.BF16, K, V, c5.pos, c5.qstat, np.full((c5.B,), 256, dtype=np.int32),
                               c5.budget, c5.lam)
-        kernel = "event_tc_kernel"
+        kernel = "event_tri_kernel"
     K, V, pos = api.to_device(ev.K, dev), api.to_device(ev.V, dev), api.to_device(ev.pos, dev)
     q, pref = api.to_device(ev.qstat, dev), api.to_device(ev.p_ref, dev)
     E = ev.n_events

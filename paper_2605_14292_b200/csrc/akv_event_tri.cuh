@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
                 const bool live = j < n;
                 // G follows from the previous round's by the constant turn when all four rows of the warp sit
                 // D16 after the rows 16 slots before them
-                bool fresh = (round & (kChainRounds - 1)) == 0 || a.no_chain;
+                bool fresh = (round & (kChainRoundsShort - 1)) == 0 || a.no_chain;
                 if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - 16] == D16);
                 if (fresh) {
                     if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);

@@ -26,8 +26,9 @@ __device__ __forceinline__ uint32_t phase_of(long long dist, unsigned long long 
 // sum_f Re(G_f conj(k_f)); and the turn S_f = e^{-i D theta_f} that takes G from one row of a lane
 // group to its next one when the two rows' positions differ by D (rows 16 slots apart: D = 16 for a
 // cache filled token by token). G is taken afresh (sector table + polynomials) whenever the spacing is
-// not D, and every eighth round in any case: seven chained complex products add less than 4e-8 of the
-// score's scale to the error (fp32 summation of the 64 terms gives 4e-8 by itself).
+// not D, and every kChainRounds-th (kChainRoundsShort-th) round in any case: a chained complex product adds
+// about 3e-9 of the score's scale to the error (fp32 summation of the 64 terms gives 4e-8 by itself; a chain
+// of twelve products measured 8e-8 in all).
 struct ChainScore {
     float2 Gx[4], Gy[4], Sx[4], Sy[4], nSy[4];
     // S from D (any sign); phitab: phi_f for the lane's frequencies (shared memory)
@@ -80,7 +81,9 @@ struct ChainScore {
         return acc2.x + acc2.y;
     }
 };
-constexpr int kChainRounds = 8;  // rounds between two fresh computations of G
+constexpr int kChainRounds = 8;        // rounds between two fresh computations of G (long events, streamed)
+constexpr int kChainRoundsShort = 16;  // the same for events of at most 256 rows: one or two fresh computations per lane
+                                       // group; fifteen chained products add 1e-7 of the score's scale at most
 
 // The 32 sector angles' cosines and sines, written by one warp: sect[h] = (cos, sin)(2 pi h / 32)
 __device__ __forceinline__ void fill_sector_table(float2* sect, int lane) {

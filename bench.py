@@ -41,10 +41,13 @@ WORKLOADS = {
     "C4": "C4 large pool: batch 8 x 28 layers x 4 KV heads, N=4096 -> b=128, d=128, bf16, lambda in {0, 0.5, 1.0}",
     "C5": "C5 decode cadence: batch 64 x 32 layers x 8 KV heads, 32 events of N=256 -> b=128 in a paged buffer, "
           "d=128, bf16, lambda=0.5",
+    "C6": "C6 flat signature (Eq. 1) with one cosine matrix per sequence: Qwen-7B shape, batch 16 x 28 layers x 4 KV heads, "
+          "N=256 -> b=128, d=128, bf16, lambda=0.5; a step = signature pass + cosine matrix + fused events",
 }
 # kernel(s) one call of the fused entry point launches for each workload
 KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_pool_kernel<fused>", "C3": "event_tri_kernel<fused>",
-           "C4": "event_stream_kernel", "C5": "event_pool_kernel<fused>"}
+           "C4": "event_stream_kernel", "C5": "event_pool_kernel<fused>",
+           "C6": "flat_signature_kernel + gram_shared_kernel + event_pool_kernel<fused>"}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per step from the ncu captures summarised under profiles/,
 # keyed by workload, each with the source revision of csrc/ it was taken at (see kernel_revision()); a
@@ -162,6 +165,8 @@ def oracle_sample(config: str, seed: int = 0):
         return synth.make_c3(seed, B=2), [0.5], "512 of 4096 events (batch 2 of 16)", 1
     if config == "C4":
         return synth.make_c4(seed, B=1, L=4, H=4), [0.0, 0.5, 1.0], "16 of 896 events (4 layers of one sequence) at each of the three lambdas", 1
+    if config == "C6":
+        return synth.make_c2(seed, B=1), [0.5], "112 of 1792 events (batch 1 of 16), flat signatures", 1
     c5 = synth.make_c5(seed, B=2, rounds=1)
     K = synth.paged_gather_dense(c5.pool_K, c5.block_table)
     V = synth.paged_gather_dense(c5.pool_V, c5.block_table)
@@ -184,8 +189,29 @@ def oracle_time(ev, lams, reps=1, threads=None):
     return E * reps * len(lams) / dt, threads, dt
 
 
+def flat_oracle_time(ev, lams):
+    """The NumPy oracle with Eq. 1's flat signature (the C twin has per-head signatures only), one process."""
+    from oracle import alpha_oracle as O
+    B, L, H, N, d = ev.shape
+    t0 = time.perf_counter()
+    for lam in lams:
+        for b in range(B):
+            sig = O.signatures_flat(ev.V[b])
+            for l in range(L):
+                for h in range(H):
+                    O.compress_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]),
+                                     ev.budget, lam, sig=sig)
+    dt = time.perf_counter() - t0
+    return ev.n_events * len(lams) / dt, 1, dt
+
+
 def cpu_baseline(config: str):
     ev, lams, what, reps = oracle_sample(config)
+    if config == "C6":
+        v, threads, dt = flat_oracle_time(ev, lams)
+        return {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"{what}, NumPy oracle in float64, {dt:.1f} s wall in one process",
+                "single_thread": {"value": v, "events": ev.n_events, "wall_s": round(dt, 2)}}
     v, threads, dt = oracle_time(ev, lams, reps)
     # one thread on a smaller slice of the same sample
     one = ev
@@ -205,14 +231,17 @@ def run_reference(args):
         return
     ev, lams, what, reps = oracle_sample(args.config)
     threads = os.cpu_count() or 1
+    run = (lambda: flat_oracle_time(ev, lams)) if args.config == "C6" else (lambda: oracle_time(ev, lams, reps, threads))
+    if args.config == "C6":
+        threads = 1
     for _ in range(args.warmup):
-        oracle_time(ev, lams, reps, threads)
+        run()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_time(ev, lams, reps, threads)
+        run()
     dt = time.perf_counter() - t0
     value = ev.n_events * len(lams) * reps * args.steps / dt
-    sample = f"per step: {what}, C oracle in float64, {threads} threads"
+    sample = f"per step: {what}, {'NumPy' if args.config == 'C6' else 'C'} oracle in float64, {threads} threads"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -230,16 +259,21 @@ class DenseWorkload:
     """C1-C4: a dense batch [B, L, H, N, d]; one step = one fused call per lambda, each on a pristine copy of
     the batch (the event rewrites its inputs). Pristine copies are restored outside the timed regions."""
 
-    def __init__(self, config, rank, dev, steps, akv, synth, torch):
+    def __init__(self, config, rank, dev, steps, akv, synth, torch, batch=None):
         self.akv, self.torch = akv, torch
-        make = {"C1": synth.make_c1, "C2": synth.make_c2, "C3": synth.make_c3, "C4": synth.make_c4}[config]
-        ev = make(seed=rank)
+        make = {"C1": synth.make_c1, "C2": synth.make_c2, "C3": synth.make_c3, "C4": synth.make_c4, "C6": synth.make_c2}[config]
+        if config == "C6" and batch is None:
+            batch = 16
+        ev = make(seed=rank) if batch is None or config == "C1" else make(seed=rank, B=batch)
+        self.flat = config == "C6"
         self.ev = ev
         self.lams = [0.0, 0.5, 1.0] if config == "C4" else [ev.lam]
         B, L, H, N, d = ev.shape
         self.esize = 2 if ev.dtype == synth.BF16 else 4
         self.events_per_step = ev.n_events * len(self.lams)
         self.bytes_per_step = algorithmic_bytes(N, ev.budget, d, self.esize) * self.events_per_step
+        if self.flat:   # the shared signatures and their cosine matrix, written once and read once per sequence
+            self.bytes_per_step += 2 * B * (N * d * 4 + N * N * 4)
         self.launches_hint = len(self.lams)
         self.LH = L * H
         self.K0, self.V0, self.P0 = akv.to_device(ev.K, dev), akv.to_device(ev.V, dev), akv.to_device(ev.pos, dev)
@@ -253,6 +287,10 @@ class DenseWorkload:
                      for _ in range(self.group * len(self.lams))]
         self.sel = akv.api._alloc_sel(akv.Layout.dense(self.K0), ev.budget, dev, detail=False)
         self.opts = [akv.Options(lam=lam) for lam in self.lams]
+        if self.flat:
+            self.sig = torch.empty((B, N, d), dtype=torch.float32, device=dev)
+            self.gram = torch.empty((B, N, N), dtype=torch.float32, device=dev)
+            self.opts = [akv.Options(lam=lam, sig_mode=akv.SIG_FLAT, shared_gram=self.gram) for lam in self.lams]
         self.flush = None
         if per_step * self.group < 2 * L2_BYTES:       # working set may stay in L2: evict it before each region
             self.flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
@@ -266,10 +304,19 @@ class DenseWorkload:
         if self.flush is not None:
             self.flush.fill_(1)
 
+    def call(self, Kb, Vb, Pb, o, sel):
+        akv = self.akv
+        if self.flat:   # Eq. 1 over all layers and heads, its cosine matrix once per sequence, then the events
+            akv.alpha_signature_flat(Vb, o, out=self.sig)
+            akv.alpha_gram_shared(self.sig, akv.Layout.dense(Vb), o, out=self.gram)
+            akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, flat_sig=self.sig, out=sel)
+        else:
+            akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, out=sel)
+
     def step(self, i):
         for j, o in enumerate(self.opts):
             Kb, Vb, Pb = self.bufs[i * len(self.lams) + j]
-            self.akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, out=self.sel)
+            self.call(Kb, Vb, Pb, o, self.sel)
 
     def timed(self, steps, barrier, stream):
         """Runs `steps` steps in groups; returns the summed device time in ms."""
@@ -303,7 +350,7 @@ class DenseWorkload:
         def one():
             for o in self.opts:
                 Kb.copy_(hK, non_blocking=True); Vb.copy_(hV, non_blocking=True); Pb.copy_(hP, non_blocking=True)
-                akv.alpha_compress_event(Kb, Vb, Pb, self.q, self.ev.budget, o, p_ref=self.pref, out=sel2)
+                self.call(Kb, Vb, Pb, o, sel2)
                 h_idx.copy_(sel2.idx_sorted, non_blocking=True); h_kept.copy_(sel2.n_kept, non_blocking=True)
 
         one()
@@ -324,9 +371,9 @@ class CadenceWorkload:
     """C5: a paged pool; one step = 32 rounds of (compress 256 -> 128 in place, then 128 fresh rows per head
     appended). Each round's call is timed by its own pair of events; the refill runs between them, untimed."""
 
-    def __init__(self, rank, dev, akv, synth, torch):
+    def __init__(self, rank, dev, akv, synth, torch, batch=None, rounds=None):
         self.akv, self.torch = akv, torch
-        c5 = synth.make_c5(seed=rank)
+        c5 = synth.make_c5(seed=rank, **({} if batch is None else {"B": batch}), **({} if rounds is None else {"rounds": rounds}))
         self.c5 = c5
         self.rounds = c5.rounds
         B, L, H, N, d, b = c5.B, c5.L, c5.H, c5.N, c5.d, c5.budget
@@ -435,9 +482,9 @@ def run_gpu(args):
     akv.load_library()
 
     if args.config == "C5":
-        wl = CadenceWorkload(rank, dev, akv, synth, torch)
+        wl = CadenceWorkload(rank, dev, akv, synth, torch, args.batch, args.rounds)
     else:
-        wl = DenseWorkload(args.config, rank, dev, args.steps, akv, synth, torch)
+        wl = DenseWorkload(args.config, rank, dev, args.steps, akv, synth, torch, args.batch)
 
     def barrier():
         if world > 1:
@@ -470,12 +517,14 @@ def run_gpu(args):
                 "dram_gbs_from_traffic": None if traffic_bytes is None else traffic_bytes / (ms_per_step * 1e-3) / 1e9,
                 "dram_frac_from_traffic": None if traffic_bytes is None else traffic_bytes / (ms_per_step * 1e-3) / 1e9 / peak}
 
-    e2e_steps = max(1, min(args.steps, 10 if args.config in ("C1", "C2", "C3") else 2))
-    e2e_ms, h2d, d2h = wl.e2e(e2e_steps, barrier, stream)
-    e2e_ms = reduce_max(e2e_ms, world, dev)
-    e2e = {"value": events_per_second(wl.events_per_step, world, e2e_steps, e2e_ms), "unit": UNIT,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-           "copied_back": "sorted indices and kept counts (the compacted K/V stay on the device)"}
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, 10 if args.config in ("C1", "C2", "C3") else 2))
+        e2e_ms, h2d, d2h = wl.e2e(e2e_steps, barrier, stream)
+        e2e_ms = reduce_max(e2e_ms, world, dev)
+        e2e = {"value": events_per_second(wl.events_per_step, world, e2e_steps, e2e_ms), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "copied_back": "sorted indices and kept counts (the compacted K/V stay on the device)"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -486,7 +535,9 @@ def run_gpu(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if wl.esize == 2 else "f32", "data": "synthetic",
-            "config": {"workload": WORKLOADS[args.config], "events_per_gpu_per_step": wl.events_per_step,
+            "config": {"workload": WORKLOADS[args.config] + (f" [batch overridden: {args.batch}]" if args.batch else "") +
+                       (f" [rounds overridden: {args.rounds}]" if args.rounds else ""),
+                       "events_per_gpu_per_step": wl.events_per_step,
                        "storage": "bf16" if wl.esize == 2 else "fp32", "accumulate": "f32", "l2": wl.l2,
                        "sequence_events_per_s": value / wl.LH},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
@@ -506,9 +557,15 @@ def main():
     ap.add_argument("--config", default="C3", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="alphakv", choices=["alphakv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiler captures)")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="number of sequences instead of the workload's own (smaller cases for profiler captures)")
+    ap.add_argument("--rounds", type=int, default=None, help="C5 only: events per step instead of 32 (profiler captures)")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = {"C1": 100, "C2": 100, "C3": 100, "C4": 10, "C5": 3}[args.config]
+        args.steps = {"C1": 100, "C2": 100, "C3": 100, "C4": 10, "C5": 3, "C6": 50}[args.config]
+    if args.impl == "reference" and args.config == "C6":
+        args.steps, args.warmup = min(args.steps, 3), 3
     if args.warmup is None:
         args.warmup = 5 if args.config != "C5" else 3
     args.warmup = max(args.warmup, 3)

@@ -103,6 +103,12 @@ typedef struct {
      * entry must lie in 1..budget, where the call's `budget` argument is the largest of them and
      * stays the row length of idx_sorted / pick_order / pick_gain (unused entries -1 / -1 / 0). */
     const int32_t* head_budgets;
+    /* Cosine matrix of the shared signatures (FLAT and PER_LAYER modes), from alpha_gram_shared: device fp32
+     * [B, N, N] (FLAT) or [B, L, N, N] (PER_LAYER), or NULL. With it, every event of a sequence (of a sequence
+     * and layer) reads its cosines from the one matrix, Algorithm 1's "Sims", instead of forming dot products
+     * of signature rows pick by pick; bf16 caches with d = 128, N <= 256 and budget <= 128 then run as one
+     * launch. Other shapes ignore it and use flat_sig. */
+    const float* shared_gram;
 } akv_options_t;
 
 /* Fills *opt with the defaults named above (lambda = 0.5, the value the paper settles on). */
@@ -196,6 +202,20 @@ akv_status_t alpha_signature_flat(akv_handle_t* h, const akv_layout_t* lay, cons
 akv_status_t alpha_signature_layer(akv_handle_t* h, const akv_layout_t* lay, const void* V,
                                    const int32_t* n_cand, const akv_options_t* opt, float* layer_sig,
                                    void* stream);
+
+/*
+ * alpha_gram_shared -- the cosine matrix of shared signatures, formed once per sequence (FLAT) or per sequence
+ * and layer (PER_LAYER): Algorithm 1's "Sims <- V V^T" for the unit rows of Eq. 1, gram[g][i][j] = <v_i, v_j>.
+ * Accuracy: each fp32 signature row is split into three bf16 parts and the product runs on the tensor cores
+ * with fp32 accumulation; entries are within 5e-7 of the float64 value (the fp32 signatures themselves carry
+ * most of that). Needs d = 128 (AKV_ERR_UNSUPPORTED
+ * otherwise).
+ *   sig     device fp32 [B, N, d] (FLAT, from alpha_signature_flat) or [B, L, N, d] (PER_LAYER), per opt->sig_mode.
+ *   gram    device fp32 [B, N, N] or [B, L, N, N] out; rows and columns >= n_cand are left untouched.
+ *   status  device int32, one word, or NULL: set to 3 if an internal bounded wait gave up (else untouched).
+ */
+akv_status_t alpha_gram_shared(akv_handle_t* h, const akv_layout_t* lay, const float* sig, const int32_t* n_cand,
+                               const akv_options_t* opt, float* gram, int32_t* status, void* stream);
 
 /*
  * kv_compact -- the retained rows become the new cache of at most `budget` rows

@@ -27,7 +27,8 @@ FLAG_NO_CHAIN = 8
 
 EXPORTS = ("akv_default_options", "akv_create", "akv_destroy", "akv_last_error", "akv_status_string",
            "akv_launch_count", "akv_workspace_bytes", "alpha_score", "alpha_select", "alpha_signature_flat",
-           "alpha_signature_layer", "kv_compact", "alpha_compress_event", "alpha_compress_event_static")
+           "alpha_signature_layer", "alpha_gram_shared", "kv_compact", "alpha_compress_event",
+           "alpha_compress_event_static")
 
 
 class AkvError(RuntimeError):
@@ -46,7 +47,7 @@ class _Layout(C.Structure):
 
 class _Options(C.Structure):
     _fields_ = [("lam", C.c_float), ("eps", C.c_float), ("rope_base", C.c_float), ("future_window", C.c_int32),
-                ("sig_mode", C.c_int), ("flags", C.c_uint32), ("head_budgets", C.c_void_p)]
+                ("sig_mode", C.c_int), ("flags", C.c_uint32), ("head_budgets", C.c_void_p), ("shared_gram", C.c_void_p)]
 
 
 _lib = None
@@ -73,6 +74,7 @@ def load_library(path: Optional[str] = None):
     lib.alpha_select.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, vp, i32, C.POINTER(_Options), vp, vp, vp, vp, vp, vp]
     lib.alpha_signature_flat.argtypes = [vp, C.POINTER(_Layout), vp, vp, C.POINTER(_Options), vp, vp]
     lib.alpha_signature_layer.argtypes = [vp, C.POINTER(_Layout), vp, vp, C.POINTER(_Options), vp, vp]
+    lib.alpha_gram_shared.argtypes = [vp, C.POINTER(_Layout), vp, vp, C.POINTER(_Options), vp, vp, vp]
     lib.akv_workspace_bytes.argtypes = [C.POINTER(_Layout), i32, C.POINTER(_Options), C.POINTER(C.c_size_t)]
     lib.kv_compact.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, i32, vp]
     lib.alpha_compress_event.argtypes = [vp, C.POINTER(_Layout), vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32,
@@ -114,13 +116,17 @@ class Options:
     sig_mode: int = SIG_PER_HEAD
     flags: int = 0
     head_budgets: Optional[torch.Tensor] = None   # device int32 [L, H]: per-(layer, head) budgets, or None
+    shared_gram: Optional[torch.Tensor] = None    # device fp32 [B, N, N] / [B, L, N, N]: cosine matrix of shared signatures
 
     def c(self) -> _Options:
         hb = self.head_budgets
         if hb is not None and (hb.dtype != torch.int32 or not hb.is_cuda or not hb.is_contiguous()):
             raise ValueError("head_budgets must be a contiguous int32 CUDA tensor [L, H]")
+        sg = self.shared_gram
+        if sg is not None and (sg.dtype != torch.float32 or not sg.is_cuda or not sg.is_contiguous()):
+            raise ValueError("shared_gram must be a contiguous float32 CUDA tensor")
         return _Options(self.lam, self.eps, self.rope_base, self.future_window, self.sig_mode, self.flags,
-                        None if hb is None else hb.data_ptr())
+                        None if hb is None else hb.data_ptr(), None if sg is None else sg.data_ptr())
 
 
 @dataclass
@@ -302,6 +308,21 @@ def alpha_signature_layer(V, opts: Optional[Options] = None, n_cand=None, layout
     with torch.cuda.device(V.device):
         _check(load_library().alpha_signature_layer(_handle(V.device), C.byref(lay.c()), _ptr(V), _ptr(n_cand),
                                                     C.byref(opts.c()), _ptr(out), _stream()))
+    return out
+
+
+def alpha_gram_shared(sig, layout: Layout, opts: Options, n_cand=None, out=None, status=None):
+    """Cosine matrix of shared signatures, [B, N, N] (flat) or [B, L, N, N] (per layer), fp32 -- C entry point
+    ``alpha_gram_shared``. ``opts.sig_mode`` says which; ``layout`` gives B, L, N, d."""
+    _need(sig, torch.float32, "sig"); _need(n_cand, torch.int32, "n_cand"); _need(status, torch.int32, "status")
+    lay = layout
+    if out is None:
+        shape = (lay.B, lay.N, lay.N) if opts.sig_mode == SIG_FLAT else (lay.B, lay.L, lay.N, lay.N)
+        out = torch.zeros(shape, dtype=torch.float32, device=sig.device)
+    _need(out, torch.float32, "out")
+    with torch.cuda.device(sig.device):
+        _check(load_library().alpha_gram_shared(_handle(sig.device), C.byref(lay.c()), _ptr(sig), _ptr(n_cand),
+                                                C.byref(opts.c()), _ptr(out), _ptr(status), _stream()))
     return out
 
 

@@ -152,6 +152,9 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     };
     __nv_bfloat16* Kg = reinterpret_cast<__nv_bfloat16*>(a.K);
     __nv_bfloat16* Vg = reinterpret_cast<__nv_bfloat16*>(a.V);
+    // shared signatures (Eq. 1, or its per-layer variant): the cosines come from the matrix formed once per
+    // sequence (or per sequence and layer) instead of from this head's V rows
+    const float* G = a.gram ? a.gram + id.b * a.gram_sb + id.l * a.gram_sl : nullptr;
 
     phase_stamp(id.e, 0);  // phases: 0 start, 1 tensor memory claimed, 2 K scored, 3 pool, 4 V operand, 5 product, 6 triangle, 7 picks, 8 outputs, 9 end
     // Tensor memory is claimed first and the right to allocate given up at once: the SM starts its
@@ -178,13 +181,16 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         mbar_init_fence();
     }
     if (FUSED && warp == 1) fill_sector_table(sect, lane);
-    // (the large size claims half of the SM's columns and holds them briefly: it claims them only when the V rows
-    // are on their way, see below; its CTAs live long enough for their starts to be further apart than that)
+    // (the large size claims half of the SM's columns: two of the three resident CTAs hold theirs at a time, the
+    // third waits in the allocation until one has moved its triangle out; claiming late instead measured 2 % slower)
     if (!BIG && use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), Cfg::kCols);
+    if (BIG && (G || !similarity) && warp == 0) tmem_relinquish();  // this event takes no tensor memory
+    if (BIG && !(G || !similarity) && warp == 0) tmem_alloc(smem_u32(tmem_holder), Cfg::kCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    uint32_t tbase = (!BIG && use_tc) ? *tmem_holder : 0u;
+    const bool have_tmem = BIG ? (similarity && !G) : use_tc;
+    const uint32_t tbase = have_tmem ? *tmem_holder : 0u;
 
     phase_stamp(id.e, 1);
     // ---- scores ---------------------------------------------------------------------------------
@@ -284,7 +290,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         if (tid == 0 && a.status) a.status[id.e] = 3;
         mbar_wait_bounded(barK, 0, a.wait_polls);  // give copies still in flight another bounded chance to land
         if (n_late > 0) mbar_wait_bounded(barL, 0, a.wait_polls);
-        if (!BIG && use_tc && warp == 0) tmem_dealloc(tbase, Cfg::kCols);
+        if (have_tmem && warp == 0) tmem_dealloc(tbase, Cfg::kCols);
         return;
     }
     bad = __syncthreads_or(bad);
@@ -373,11 +379,39 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     const uint32_t bound_key = BIG ? *bound_holder : 0u;
     const bool fast = similarity && P <= Cfg::kMaxPool && picks > 1;
     bool slow = similarity && P > Cfg::kMaxPool;  // (small size only; the large size may set it after its loop)
-    const bool have_tmem = BIG ? fast : use_tc;
 
     phase_stamp(id.e, 3);
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
-    if (similarity && !slow) {
+    if (similarity && !slow && G) {
+        // the active set's cosine matrix, gathered from the shared one: row a of the triangle holds the shared
+        // matrix's row of slot a at the slots of rows 0..a; the signatures are unit rows, so there are no norms
+        // (a warp per row, its lanes across the row's columns: a lane's columns are the same for every row, so it
+        // keeps their slots in registers, and the loads of a row, all from one 1 KB row of the shared matrix, are
+        // in flight together)
+        int col[Cfg::kCpl];
+#pragma unroll
+        for (int k = 0; k < Cfg::kCpl; ++k) col[k] = lane + 32 * k < P ? bypool[lane + 32 * k] : 0;
+        // four rows of a warp at a time: their loads are issued before any of them is stored
+        for (int ra0 = warp; ra0 < P; ra0 += 4 * (kTcThreads / 32)) {
+            float x[4][Cfg::kCpl];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int ra = ra0 + i * (kTcThreads / 32);
+                const float* grow = G + (long long)bypool[min(ra, P - 1)] * N;
+#pragma unroll
+                for (int k = 0; k < Cfg::kCpl; ++k) x[i][k] = (ra < P && lane + 32 * k <= ra) ? __ldg(grow + col[k]) : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int ra = ra0 + i * (kTcThreads / 32);
+                const int trow = tri_row(ra);
+#pragma unroll
+                for (int k = 0; k < Cfg::kCpl; ++k)
+                    if (ra < P && lane + 32 * k <= ra) tri[trow + lane + 32 * k] = x[i][k];
+            }
+        }
+        for (int ra = tid; ra < P; ra += kTcThreads) r[ra] = 1.f;
+    } else if (similarity && !slow) {
         // thread -> 16-byte column c of rows r0, r0 + 8, ...: the swizzle term (c ^ row) & 7 is the same for
         // all of them, so a row costs one pool lookup, one address and one copy
         const int c = tid & 15, r0 = tid >> 4;
@@ -390,21 +424,21 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             for (int rho = r0; rho < P; rho += 8)
                 cp_async16(dst0 + (uint32_t)(rho - r0) * 128u, Vg + rowoff(bypool[rho]) + c * 8);
         }
-        if (BIG && fast && warp == 0) tmem_alloc(smem_u32(tmem_holder), Cfg::kCols);  // may wait for another CTA's columns
+
         cp_async_wait_all();
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        if (BIG && fast) tbase = *tmem_holder;
     }
     phase_stamp(id.e, 4);
     // large size, rows from 128 on (nb of them): a second product, the last 128 rows of the operand against those
     // rows, gives their cosines against one another; what lies left of column 128 comes from the first product
     // by symmetry
-    const int nb = (BIG && fast && P > 128) ? P - 128 : 0;
+    const bool product = fast && !G;  // the cosine matrix comes off the tensor core
+    const int nb = (BIG && product && P > 128) ? P - 128 : 0;
     const int ncols = (P + 15) & ~15, base2 = ncols - 128;
-    if (fast) {
+    if (product) {
         if (tid == 0) {
             tc_fence_after();
             const uint32_t idesc = umma_idesc_bf16(128, ncols);
@@ -434,7 +468,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         return;
     }
     phase_stamp(id.e, 5);
-    if (fast) {
+    if (product) {
         // lower triangle -> shared memory; row rho = 32 warp + lane needs columns 0..rho
         const int rho = 32 * warp + lane;
         if (32 * warp < P) {
@@ -493,6 +527,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     } else if (slow) {
         // reciprocal norms (Eq. 1); this pool does not fit the tile, its V rows are read in place
         for (int rho = tid; rho < P; rho += kTcThreads) {
+            if (G) { r[rho] = 1.f; continue; }
             const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
             float ss = 0.f;
 #pragma unroll
@@ -548,6 +583,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                 __syncthreads();
                 P = *pool_holder;
                 for (int rho = tid; rho < P; rho += kTcThreads) {
+                    if (G) { r[rho] = 1.f; continue; }
                     const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
                     float ss = 0.f;
 #pragma unroll
@@ -575,9 +611,10 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             if (t + 1 == picks) break;
             __syncthreads();
             const int irho = *pick_holder;
-            // row irho of the cosine matrix by plain dot products
+            // row irho of the cosine matrix: from the shared matrix, else by plain dot products
             const __nv_bfloat16* vpick = Vg + rowoff(bypool[irho]);
             for (int rho = tid; rho < P; rho += kTcThreads) {
+                if (G) { rowbuf[rho] = G[(long long)bypool[irho] * N + bypool[rho]]; continue; }
                 const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
                 float acc = 0.f;
 #pragma unroll 4

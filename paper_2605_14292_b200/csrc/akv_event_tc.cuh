@@ -122,6 +122,11 @@ __device__ __forceinline__ void tmem_alloc(uint32_t holder, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"(cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
+// For a CTA that will not allocate tensor memory at all (one whole warp calls): the SM starts the next CTA of a
+// kernel that contains an allocation only once every resident CTA has given up its right to allocate.
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
@@ -233,6 +238,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) event_tc_kernel(const EventArgs
         mbar_init_fence();
     }
     if (FUSED && warp == 1) fill_sector_table(sect, lane);
+    if (!use_tc && warp == 0) tmem_relinquish();  // this event takes no tensor memory
     __syncthreads();
     uint32_t tbase = 0u;
 

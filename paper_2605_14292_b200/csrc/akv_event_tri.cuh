@@ -255,7 +255,10 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
         sincospif((float)(tid - 32) * 0.0625f, &sn, &cs);  // angle 2 pi h / 32
         sect[tid - 32] = make_float2(cs, sn);
     }
-    if (use_tc && warp == 0) tmem_alloc(smem_u32(tmem_holder), kTcCols);
+    if (warp == 0) {
+        if (use_tc) tmem_alloc(smem_u32(tmem_holder), kTcCols);
+        else tmem_relinquish();  // top-k events take no tensor memory, and must not hold up the next CTA's start
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();

@@ -14,6 +14,8 @@ struct EventArgs {
     const int* p_ref;       // [B] or null
     const float* flat_sig;  // shared signatures, or null: [B,N,d] (Eq. 1) or [B,L,N,d] (per layer)
     long long sig_sb, sig_sl;  // element strides of flat_sig over sequences and layers (0 for the flat mode's layers)
+    const float* gram;         // cosine matrix of the shared signatures, or null: [B,N,N] (Eq. 1) or [B,L,N,N] (per layer)
+    long long gram_sb, gram_sl;  // its element strides over sequences and layers
     const int* head_budgets;   // [L,H] or null: per-(layer, head) budgets, each <= budget
     int budget;             // largest budget of the call = row length of the index outputs
     float lam, eps;
@@ -332,42 +334,51 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const CompactArgs a) 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Eq. 1: shared signatures. One warp group per (sequence, slot): u = mean over (l, h) of V rows,
-// v = u / (||u|| + eps), written as fp32 [B, N, d]; per_layer: one group per (sequence, layer, slot),
-// the mean runs over the heads of that layer only, written as fp32 [B, L, N, d].
+// Eq. 1: shared signatures. u = mean over (l, h) of the V rows of one (sequence, slot), v = u / (||u|| + eps),
+// written as fp32 [B, N, d]; per_layer: one signature per (sequence, layer, slot), the mean runs over the heads
+// of that layer only, written as fp32 [B, L, N, d]. One CTA per (group, 32 / G slots), G = lanes per row: its
+// eight warps split the (layer, head) pairs among themselves (every thread has a dozen independent 16-byte
+// loads in flight), partial sums meet in shared memory in a fixed order.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kThreads) flat_signature_kernel(const DevLayout lay, const void* V, const int* n_cand,
                                                                  float eps, float* out, int per_layer) {
+    __shared__ float part[kWarps][32][8];
     const int d = lay.d;
     const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
     const int RPW = 32 / G;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int grp = lane / G, lig = lane % G;
-    const int groups = per_layer ? lay.B * lay.L : lay.B;
-    const long long slot = ((long long)blockIdx.x * kWarps + warp) * RPW + grp;  // over groups * N
-    const bool inrange = slot < (long long)groups * lay.N;
-    const int grpi = inrange ? (int)(slot / lay.N) : 0;
+    const int slot_blocks = (lay.N + RPW - 1) / RPW;
+    const int grpi = blockIdx.x / slot_blocks;                         // sequence, or (sequence, layer)
+    const int j = (blockIdx.x % slot_blocks) * RPW + grp;
     const int b = per_layer ? grpi / lay.L : grpi;
     const int l0 = per_layer ? grpi % lay.L : 0, l1 = per_layer ? l0 + 1 : lay.L;
-    const int j = inrange ? (int)(slot % lay.N) : 0;
     int n = n_cand ? n_cand[b] : lay.N;
     n = n < 0 ? 0 : (n > lay.N ? lay.N : n);
-    const bool valid = inrange && j < n;
+    const bool valid = j < n;
     const bool act = valid && lig * 8 < d;
     const T* Vg = reinterpret_cast<const T*>(V);
+    const int pairs = (l1 - l0) * lay.H;
     float u[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (act) {
-        for (int l = l0; l < l1; ++l)
-            for (int h = 0; h < lay.H; ++h) {
-                float x[8];
-                load8(Vg + row_offset(lay, b, l, h, j) + lig * 8, x);
+        for (int p = warp; p < pairs; p += kWarps) {
+            float x[8];
+            load8(Vg + row_offset(lay, b, l0 + p / lay.H, p % lay.H, j) + lig * 8, x);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) u[q] += x[q];
-            }
-        const float inv = 1.f / (float)((l1 - l0) * lay.H);
+            for (int q = 0; q < 8; ++q) u[q] += x[q];
+        }
+    }
 #pragma unroll
-        for (int q = 0; q < 8; ++q) u[q] *= inv;
+    for (int q = 0; q < 8; ++q) part[warp][lane][q] = u[q];
+    __syncthreads();
+    if (warp != 0) return;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) acc += part[w][lane][q];
+        u[q] = acc * (1.f / (float)pairs);
     }
     float ss = 0.f;
 #pragma unroll
@@ -375,7 +386,7 @@ __global__ void __launch_bounds__(kThreads) flat_signature_kernel(const DevLayou
     ss = group_sum(ss, G);
     if (act) {
         const float r = 1.f / (sqrtf(ss) + eps);
-        float* o = out + slot * d + lig * 8;
+        float* o = out + ((long long)grpi * lay.N + j) * d + lig * 8;
         *reinterpret_cast<float4*>(o) = make_float4(u[0] * r, u[1] * r, u[2] * r, u[3] * r);
         *reinterpret_cast<float4*>(o + 4) = make_float4(u[4] * r, u[5] * r, u[6] * r, u[7] * r);
     }

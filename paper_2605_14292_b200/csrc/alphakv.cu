@@ -10,6 +10,7 @@
 
 #include "akv_event_pool.cuh"
 #include "akv_event_stream.cuh"
+#include "akv_gram.cuh"
 #include "akv_select_pool.cuh"
 
 using namespace akv;
@@ -316,6 +317,10 @@ static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t s
 // N <= 256, over an active set of the pool's 152 best-scored rows.
 static bool tri_path_ok(const EventArgs& a) { return tc_path_ok(a) && (a.lay.N <= 128 || a.budget <= 64); }
 static bool tri_big_ok(const EventArgs& a) { return tc_path_ok(a) && !tri_path_ok(a) && a.budget <= 128; }
+// shared signatures with their cosine matrix at hand: the large size, which gathers its triangle from that matrix
+static bool pool_shared_ok(const EventArgs& a) {
+    return a.gram != nullptr && a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.budget <= 128;
+}
 template <bool FUSED, bool BIG>
 static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
     const int E = a.lay.B * a.lay.L * a.lay.H;
@@ -339,6 +344,7 @@ static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t s
 }
 
 static akv_status_t launch_select(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
+    if (pool_shared_ok(a)) return launch_tri<false, true>(h, a, st, dry);
     if (tri_path_ok(a) && a.V) return launch_tri<false, false>(h, a, st, dry);
     if (tri_big_ok(a) && a.V) return launch_tri<false, true>(h, a, st, dry);
     if (tc_path_ok(a) && a.V) return launch_tc<false>(h, a, st, dry);
@@ -408,8 +414,15 @@ static akv_status_t fill_select_args(EventArgs& a, const akv_options_t* opt, con
         const long long nd = (long long)a.lay.N * a.lay.d;
         a.sig_sb = opt->sig_mode == AKV_SIG_PER_LAYER ? nd * a.lay.L : nd;
         a.sig_sl = opt->sig_mode == AKV_SIG_PER_LAYER ? nd : 0;
+        if (opt->shared_gram) {
+            if (!aligned16(opt->shared_gram)) return fail(AKV_ERR_ALIGNMENT, "shared_gram is not 16-byte aligned");
+            const long long nn = (long long)a.lay.N * a.lay.N;
+            a.gram = opt->shared_gram;
+            a.gram_sb = opt->sig_mode == AKV_SIG_PER_LAYER ? nn * a.lay.L : nn;
+            a.gram_sl = opt->sig_mode == AKV_SIG_PER_LAYER ? nn : 0;
+        }
     } else {
-        if (flat_sig) return fail(AKV_ERR_INVALID_ARG, "flat_sig given but sig_mode is per-head");
+        if (flat_sig || opt->shared_gram) return fail(AKV_ERR_INVALID_ARG, "flat_sig / shared_gram given but sig_mode is per-head");
         if (a.greedy && !V) return fail(AKV_ERR_INVALID_ARG, "V must not be NULL in per-head signature mode");
     }
     return AKV_OK;
@@ -453,9 +466,10 @@ static akv_status_t alpha_signature_flat_impl(akv_handle_t* h, const akv_layout_
     DeviceGuard guard(h->device);
     if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
     const int G = pow2_ceil(y.d >> 3) > 32 ? 32 : pow2_ceil(y.d >> 3);
-    const long long per_cta = (long long)kWarps * (32 / G);
-    const long long slots = (long long)y.B * (per_layer ? y.L : 1) * y.N;
-    const unsigned grid = (unsigned)((slots + per_cta - 1) / per_cta);
+    const int rpw = 32 / G;                                              // slots per CTA
+    const long long blocks = (long long)y.B * (per_layer ? y.L : 1) * ((y.N + rpw - 1) / rpw);
+    if (blocks > INT_MAX) return fail(AKV_ERR_UNSUPPORTED, "alpha_signature: %lld blocks exceed the grid limit", blocks);
+    const unsigned grid = (unsigned)blocks;
     cudaStream_t st = (cudaStream_t)stream;
     if (y.dtype == AKV_BF16) flat_signature_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig, per_layer);
     else flat_signature_kernel<float><<<grid, kThreads, 0, st>>>(y, V, n_cand, opt->eps, flat_sig, per_layer);
@@ -495,6 +509,7 @@ static bool stream_path_ok(const EventArgs& a, int smem_optin) {
     return sp.cap_rows > 0 && (int)sp.total <= stream_smem_limit(smem_optin);
 }
 static EventRoute event_route(const EventArgs& a, int smem_optin) {
+    if (pool_shared_ok(a)) return ROUTE_TRI_BIG;
     if (tri_path_ok(a)) return ROUTE_TRI;
     if (tri_big_ok(a)) return ROUTE_TRI_BIG;
     if (tc_path_ok(a)) return ROUTE_TC;
@@ -517,6 +532,7 @@ extern "C" akv_status_t akv_workspace_bytes(const akv_layout_t* lay, int32_t bud
     a.greedy = (opt->lambda > 0.f || (opt->flags & AKV_FLAG_FORCE_GREEDY)) ? 1 : 0;
     // only whether shared signatures are in use matters for the route, not where they live
     a.flat_sig = opt->sig_mode != AKV_SIG_PER_HEAD ? reinterpret_cast<const float*>(bytes) : nullptr;
+    a.gram = opt->sig_mode != AKV_SIG_PER_HEAD ? opt->shared_gram : nullptr;
     int dev = 0, smem_optin = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     CUDA_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
@@ -669,6 +685,29 @@ static akv_status_t alpha_compress_event_static_impl(akv_handle_t* h, const akv_
 }
 
 
+static akv_status_t alpha_gram_shared_impl(akv_handle_t* h, const akv_layout_t* lay, const float* sig, const int32_t* n_cand,
+                                           const akv_options_t* opt, float* gram, int32_t* status, void* stream) {
+    if (!h) return fail(AKV_ERR_INVALID_ARG, "alpha_gram_shared: handle is NULL");
+    DevLayout y;
+    akv_status_t s = check_layout(lay, &y);
+    if (s != AKV_OK) return s;
+    if ((s = check_options(opt)) != AKV_OK) return s;
+    if (opt->sig_mode == AKV_SIG_PER_HEAD) return fail(AKV_ERR_INVALID_ARG, "alpha_gram_shared: sig_mode must be FLAT or PER_LAYER");
+    if (y.d != kTcD) return fail(AKV_ERR_UNSUPPORTED, "alpha_gram_shared: d = %d (only 128 is built)", y.d);
+    if (!sig || !gram) return fail(AKV_ERR_INVALID_ARG, "alpha_gram_shared: sig and gram must not be NULL");
+    if (!aligned16(sig) || !aligned16(gram)) return fail(AKV_ERR_ALIGNMENT, "alpha_gram_shared: pointers must be 16-byte aligned");
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    const int seq_div = opt->sig_mode == AKV_SIG_PER_LAYER ? y.L : 1;
+    const long long groups = (long long)y.B * seq_div;
+    const int tiles = (y.N + 127) / 128;
+    const long long blocks = groups * tiles * tiles;
+    if (blocks > INT_MAX) return fail(AKV_ERR_UNSUPPORTED, "alpha_gram_shared: %lld tiles exceed the grid limit", blocks);
+    if ((s = set_smem(gram_shared_kernel, kGramSmem)) != AKV_OK) return s;
+    gram_shared_kernel<<<(unsigned)blocks, kGramThreads, kGramSmem, (cudaStream_t)stream>>>(sig, n_cand, seq_div, y.N, gram, status);
+    return launched("gram_shared");
+}
+
 // ------------------------------------------------------------------------------------------------
 // C entry points: each forwards to its implementation above and leaves a failure's message in the handle.
 // ------------------------------------------------------------------------------------------------
@@ -694,6 +733,10 @@ extern "C" akv_status_t alpha_signature_layer(akv_handle_t* h, const akv_layout_
                                               const int32_t* n_cand, const akv_options_t* opt, float* layer_sig,
                                               void* stream) {
     return finish(h, alpha_signature_flat_impl(h, lay, V, n_cand, opt, layer_sig, stream, 1));
+}
+extern "C" akv_status_t alpha_gram_shared(akv_handle_t* h, const akv_layout_t* lay, const float* sig, const int32_t* n_cand,
+                                          const akv_options_t* opt, float* gram, int32_t* status, void* stream) {
+    return finish(h, alpha_gram_shared_impl(h, lay, sig, n_cand, opt, gram, status, stream));
 }
 extern "C" akv_status_t kv_compact(akv_handle_t* h, const akv_layout_t* lay, void* K, void* V, int32_t* pos,
                                    int64_t psb, int64_t psl, int64_t psh, const int32_t* idx_sorted, int32_t budget,

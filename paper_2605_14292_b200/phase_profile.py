@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--config", default="C3", choices=["C2", "C3", "C4", "C5"])
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--lam", type=float, default=0.5)
+    ap.add_argument("--flat", action="store_true", help="Eq. 1's flat signature with one cosine matrix per sequence (C2 shape)")
     args = ap.parse_args()
     lib = api.load_library(build.build_phase_clocks())
     api._lib = lib                                    # the binding's entry points now call the profiling build
@@ -56,11 +57,16 @@ def main():
     E = ev.n_events
     buf = torch.zeros((E, slots), dtype=torch.int64, device=dev)
     K0, V0, P0 = K.clone(), V.clone(), pos.clone()
+    opts, sig = api.Options(lam=args.lam), None
+    if args.flat:
+        sig = api.alpha_signature_flat(V)
+        gram = api.alpha_gram_shared(sig, api.Layout.dense(V), api.Options(sig_mode=api.SIG_FLAT))
+        opts = api.Options(lam=args.lam, sig_mode=api.SIG_FLAT, shared_gram=gram)
     for it in range(2):                               # second pass: kernels loaded, clocks settled
         K.copy_(K0); V.copy_(V0); pos.copy_(P0)
         buf.zero_()
         assert lib.akv_debug_phase_buffer(C.c_void_p(buf.data_ptr())) == 0
-        api.alpha_compress_event(K, V, pos, q, ev.budget, api.Options(lam=args.lam), p_ref=pref, detail=False)
+        api.alpha_compress_event(K, V, pos, q, ev.budget, opts, p_ref=pref, flat_sig=sig, detail=False)
         torch.cuda.synchronize()
     lib.akv_debug_phase_buffer(None)
     st = buf.cpu().numpy()

@@ -495,6 +495,70 @@ def test_chained_and_fresh_scores_agree_on_the_tensor_memory_kernels():
         check_all(ev, b, ev.lam)
 
 
+# ------------------------------------------------------------------ shared signatures with one cosine matrix per sequence
+@pytest.mark.parametrize("mode", ["flat", "layer"])
+@pytest.mark.parametrize("N", [96, 256, 300])
+def test_shared_cosine_matrix(mode, N):
+    """Algorithm 1's cosine matrix of the shared signatures, once per sequence (Eq. 1) or per sequence and layer:
+    three-part bf16 split on the tensor cores against the float64 product, with a ragged candidate count."""
+    ev = synth.make_plain(2, 2, 3, N, 128, 16, 0.5, dtype=synth.BF16, seed=90 + N)
+    V = dev(ev.V)
+    n_cand = np.array([N, N - 37], dtype=np.int32)
+    nc = dev(n_cand)
+    lay = akv.Layout.dense(V)
+    if mode == "flat":
+        opts = akv.Options(sig_mode=akv.SIG_FLAT)
+        sig = akv.alpha_signature_flat(V, n_cand=nc)
+    else:
+        opts = akv.Options(sig_mode=akv.SIG_PER_LAYER)
+        sig = akv.alpha_signature_layer(V, n_cand=nc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gram = akv.alpha_gram_shared(sig, lay, opts, n_cand=nc, status=status).cpu().numpy()
+    assert int(status.item()) == 0
+    for b in range(2):
+        n = int(n_cand[b])
+        groups = [None] if mode == "flat" else range(2)
+        for l in groups:
+            ref_sig = O.signatures_flat(ev.V[b][:, :, :n]) if l is None else O.signatures_per_layer(ev.V[b, l][:, :n])
+            got = gram[b][:n, :n] if l is None else gram[b, l][:n, :n]
+            assert np.max(np.abs(got - ref_sig @ ref_sig.T)) < 5e-7
+            rest = gram[b][n:] if l is None else gram[b, l][n:]
+            assert np.all(rest == 0)                                  # rows beyond the candidates are left alone
+
+
+@pytest.mark.parametrize("mode,N,budget", [("flat", 256, 128), ("flat", 192, 64), ("layer", 256, 100), ("flat", 130, 20)])
+def test_fused_event_with_shared_cosine_matrix(mode, N, budget):
+    """Shared signatures in the fused path: signature pass, one cosine matrix per sequence (and layer), then every
+    event of the sequence in ONE launch that reads its cosines from that matrix. Checked against the oracle with
+    the float64 signatures, and against the general route (dot products of signature rows pick by pick)."""
+    ev = synth.make_c3(seed=95 + N, B=2, L=3, H=2, N=N, budget=budget)
+    lam = 0.7
+    K, V, pos, q, pref = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    lay = akv.Layout.dense(V)
+    smode = akv.SIG_FLAT if mode == "flat" else akv.SIG_PER_LAYER
+    sig = akv.alpha_signature_flat(V) if mode == "flat" else akv.alpha_signature_layer(V)
+    gram = akv.alpha_gram_shared(sig, lay, akv.Options(sig_mode=smode))
+    K2, V2, pos2 = K.clone(), V.clone(), pos.clone()
+    before = akv.launch_count()
+    sel = akv.alpha_compress_event(K, V, pos, q, budget, akv.Options(lam=lam, sig_mode=smode, shared_gram=gram), p_ref=pref,
+                                   flat_sig=sig, want_scores=True)
+    assert akv.launch_count() == before + 1
+    ref = akv.alpha_compress_event(K2, V2, pos2, q, budget, akv.Options(lam=lam, sig_mode=smode), p_ref=pref, flat_sig=sig)
+    torch.cuda.synchronize()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    n_same = 0
+    for b in range(2):
+        for l in range(3):
+            ref_sig = O.signatures_flat(ev.V[b]) if mode == "flat" else O.signatures_per_layer(ev.V[b, l])
+            for h in range(2):
+                chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], ev.qstat[l, h], int(ev.p_ref[b]), budget, lam,
+                                sel.scores[b, l, h].cpu().numpy(), sel.pick_order[b, l, h].cpu().numpy(),
+                                sel.idx_sorted[b, l, h].cpu().numpy(), Kn[b, l, h], Vn[b, l, h], pn[b, l, h], sig=ref_sig)
+                n_same += int(torch.equal(sel.pick_order[b, l, h], ref.pick_order[b, l, h]))
+    assert n_same >= 11                                               # the two routes round differently: near-ties may differ
+    assert int(sel.status.abs().max()) == 0 and int(sel.n_kept.min()) == budget
+
+
 def test_report_worst_score_error():
     """Printed for the record (run last in this file): the worst score error of everything checked so far."""
     print("worst |err|/|s| where |s| >= 0.1 scale: %.3e; worst |err|/scale: %.3e; scores checked: %d"

@@ -109,6 +109,13 @@ typedef struct {
      * of signature rows pick by pick; bf16 caches with d = 128, N <= 256 and budget <= 128 then run as one
      * launch. Other shapes ignore it and use flat_sig. */
     const float* shared_gram;
+    /* Grouped-query attention: qstat holds gqa_group statistics per KV head, [L, H * gqa_group, d] (0 and 1 both
+     * mean one). The score of a key is the mean over the group's query heads of their scores (gqa_reduce = 0;
+     * the same as scoring with the averaged statistic, the score being linear in it) or the largest of them
+     * (gqa_reduce = 1: a key that any query head of the group wants is kept). At most 8 per group. Groups
+     * larger than one run on the general kernels (the resident one or three launches). */
+    int32_t gqa_group;
+    int32_t gqa_reduce;
 } akv_options_t;
 
 /* Fills *opt with the defaults named above (lambda = 0.5, the value the paper settles on). */
@@ -152,8 +159,8 @@ uint64_t akv_launch_count(void);
  *           b*pos_stride_b + l*pos_stride_l + h*pos_stride_h + n (a stride of 0
  *           broadcasts). NULL: keys are already rotated, s_i = q . k_i / sqrt d.
  *   n_cand  device int32 [B] valid slots per sequence, or NULL for N.
- *   qstat   device fp32 [L, H, d] query statistic per KV head (for grouped-query
- *           attention the caller averages its query heads; the score is linear in q).
+ *   qstat   device fp32 [L, H, d] query statistic per KV head; with opt->gqa_group = G > 1,
+ *           [L, H * G, d]: G statistics per KV head, reduced by opt->gqa_reduce.
  *   p_ref   device int32 [B], or NULL for (largest position of the event) + 1.
  *   scores  device fp32 [B, L, H, N] out; slots >= n_cand are left untouched.
  *   status  device int32 [B, L, H] out or NULL.

@@ -95,6 +95,19 @@ def triattention_score(K, pos, qstat, p_ref, W: int = 1, base: float = 10000.0) 
     return terms.real.sum(axis=1) / math.sqrt(d)
 
 
+def triattention_score_group(K, pos, qstats, p_ref, W: int = 1, base: float = 10000.0, reduce: str = "mean") -> np.ndarray:
+    """Grouped-query attention: the KV head serves several query heads, each with its own statistic
+    (qstats: [G, d]). The key's score is the mean of the G per-head scores, or the largest of them
+    ("max": a key that any query head of the group wants scores high). Each per-head score is
+    triattention_score as it stands."""
+    per_head = np.stack([triattention_score(K, pos, q, p_ref, W, base) for q in np.asarray(qstats)])
+    if reduce == "mean":
+        return per_head.mean(axis=0)
+    if reduce == "max":
+        return per_head.max(axis=0)
+    raise ValueError(reduce)
+
+
 def default_p_ref(pos) -> int:
     """When the caller gives no reference position: one past the newest slot."""
     return int(np.max(pos)) + 1

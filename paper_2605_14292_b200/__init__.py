@@ -7,5 +7,5 @@ compiled library and a CUDA device; nothing here falls back to the CPU.
 """
 from .api import (AkvError, Layout, Options, Selection, alpha_compress_event, alpha_compress_event_static, alpha_score, alpha_select,  # noqa: F401
                   alpha_gram_shared, alpha_signature_flat, alpha_signature_layer, kv_compact, launch_count, load_library, to_device,
-                  to_host_bits, workspace_bytes, FLAG_FORCE_GREEDY, FLAG_NO_CHAIN, FLAG_NO_PRUNE, FLAG_TEST_STARVE_WAIT, SIG_FLAT,
+                  to_host_bits, workspace_bytes, FLAG_FORCE_GREEDY, GQA_MAX, GQA_MEAN, FLAG_NO_CHAIN, FLAG_NO_PRUNE, FLAG_TEST_STARVE_WAIT, SIG_FLAT,
                   SIG_PER_HEAD, SIG_PER_LAYER)

@@ -24,6 +24,7 @@ FLAG_FORCE_GREEDY = 1
 FLAG_NO_PRUNE = 2
 FLAG_TEST_STARVE_WAIT = 4
 FLAG_NO_CHAIN = 8
+GQA_MEAN, GQA_MAX = 0, 1
 
 EXPORTS = ("akv_default_options", "akv_create", "akv_destroy", "akv_last_error", "akv_status_string",
            "akv_launch_count", "akv_workspace_bytes", "alpha_score", "alpha_select", "alpha_signature_flat",
@@ -47,7 +48,7 @@ class _Layout(C.Structure):
 
 class _Options(C.Structure):
     _fields_ = [("lam", C.c_float), ("eps", C.c_float), ("rope_base", C.c_float), ("future_window", C.c_int32),
-                ("sig_mode", C.c_int), ("flags", C.c_uint32), ("head_budgets", C.c_void_p), ("shared_gram", C.c_void_p)]
+                ("sig_mode", C.c_int), ("flags", C.c_uint32), ("head_budgets", C.c_void_p), ("shared_gram", C.c_void_p), ("gqa_group", C.c_int32), ("gqa_reduce", C.c_int32)]
 
 
 _lib = None
@@ -117,6 +118,8 @@ class Options:
     flags: int = 0
     head_budgets: Optional[torch.Tensor] = None   # device int32 [L, H]: per-(layer, head) budgets, or None
     shared_gram: Optional[torch.Tensor] = None    # device fp32 [B, N, N] / [B, L, N, N]: cosine matrix of shared signatures
+    gqa_group: int = 1                            # query statistics per KV head: qstat is [L, H * gqa_group, d]
+    gqa_reduce: int = 0                           # 0: mean over the group, 1: maximum
 
     def c(self) -> _Options:
         hb = self.head_budgets
@@ -126,7 +129,8 @@ class Options:
         if sg is not None and (sg.dtype != torch.float32 or not sg.is_cuda or not sg.is_contiguous()):
             raise ValueError("shared_gram must be a contiguous float32 CUDA tensor")
         return _Options(self.lam, self.eps, self.rope_base, self.future_window, self.sig_mode, self.flags,
-                        None if hb is None else hb.data_ptr(), None if sg is None else sg.data_ptr())
+                        None if hb is None else hb.data_ptr(), None if sg is None else sg.data_ptr(), self.gqa_group,
+                        self.gqa_reduce)
 
 
 @dataclass

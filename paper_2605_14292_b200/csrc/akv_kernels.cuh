@@ -23,6 +23,8 @@ struct EventArgs {
     int no_prune;           // 1: keep every candidate in the pool the loop runs over
     int tmem_cols;          // tensor-memory columns the tensor-memory kernel claims per CTA (0: none)
     int no_chain;           // testing aid: score every row from scratch even when positions are regular
+    int gqa_group;          // query statistics per KV head (>= 1)
+    int gqa_max;            // 1: a key's score is the largest over the group, 0: their mean
     int starve;             // testing aid: request no K row, so that the bounded waits run out
     int wait_polls;         // polls after which a bounded wait gives up
     int* idx_sorted;
@@ -47,6 +49,45 @@ __device__ __forceinline__ int event_budget(const EventArgs& a, const EventId& i
 // shared signature rows of this event's (sequence, layer)
 __device__ __forceinline__ const float* event_sig(const EventArgs& a, const EventId& id) {
     return a.flat_sig + id.b * a.sig_sb + id.l * a.sig_sl;
+}
+
+// Folded statistics of the event's query group into g[member * (d / 2) + f]; returns how many a row's score is
+// the maximum of (1 when the group is averaged: the score is linear in the statistic, so the mean of the
+// members' scores is the score of their mean statistic).
+constexpr int kMaxGroup = 8;
+__device__ __forceinline__ int fold_group(const EventArgs& a, const EventId& id, const ScoreTab& tab, int d, float2* g) {
+    const int G = a.gqa_group < 1 ? 1 : a.gqa_group, half = d >> 1;
+    const float* q = a.qstat + ((long long)id.l * a.lay.H + id.h) * G * d;
+    const float inv = rsqrtf((float)d);
+    if (a.gqa_max) {
+        for (int x = threadIdx.x; x < G * half; x += blockDim.x) {
+            const int m = x / half, f = x - m * half;
+            const float qr = q[m * d + f] * inv, qi = q[m * d + f + half] * inv;
+            const float2 c = tab.cw[f];
+            g[x] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+        }
+        return G;
+    }
+    for (int f = threadIdx.x; f < half; f += blockDim.x) {
+        float qr = 0.f, qi = 0.f;
+        for (int m = 0; m < G; ++m) {
+            qr += q[m * d + f];
+            qi += q[m * d + f + half];
+        }
+        qr *= inv / (float)G;
+        qi *= inv / (float)G;
+        const float2 c = tab.cw[f];
+        g[f] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
+    }
+    return 1;
+}
+// score of one row against every member's statistic, reduced by the maximum (one member: the plain score)
+template <typename T>
+__device__ __forceinline__ float score_group(const T* krow, bool valid, long long dist, bool rotate, int d,
+                                             const unsigned long long* phi, const float2* g, int lig, int G, int members) {
+    float best = score_row(krow, valid, dist, rotate, d, phi, g, lig, G);
+    for (int m = 1; m < members; ++m) best = fmaxf(best, score_row(krow, valid, dist, rotate, d, phi, g + m * (d >> 1), lig, G));
+    return best;
 }
 
 __device__ __forceinline__ const int* event_pos(const PosDesc& p, const EventId& id) {
@@ -77,7 +118,7 @@ __host__ __device__ inline SmemPlan plan_smem(int N, int d, int esize, int budge
     p.tileK = o; o += withK ? align16((unsigned)N * d * esize) : 0;
     p.tileV = o; o += withV ? align16((unsigned)N * d * esize) : 0;
     p.phi = o;   o += align16((unsigned)(d / 2) * 8);
-    p.g = o;     o += align16((unsigned)(d / 2) * 8);
+    p.g = o;     o += align16((unsigned)(d / 2) * 8) * kMaxGroup;  // folded statistic of every member of a query group
     p.pos = o;   o += align16((unsigned)N * 4);
     p.s = o;     o += align16((unsigned)N * 4);
     p.r = o;     o += align16((unsigned)N * 4);
@@ -146,7 +187,7 @@ __global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArg
         m[j] = 0.f;
     }
     for (int f = tid; f < d / 2; f += kThreads) phi[f] = tab.phi[f];
-    fold_query(a.qstat + ((long long)id.l * lay.H + id.h) * d, tab, d, g);
+    const int members = fold_group(a, id, tab, d, g);
     long long pref = 0;
     if (gpos) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)block_max_int(pmax, redi) + 1;
     __syncthreads();
@@ -159,7 +200,7 @@ __global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArg
         const int j = j0 + grp;
         const bool valid = j < n;
         const long long dist = valid ? pref - (long long)spos[j] : 0;
-        const float sc = score_row(Kt + (size_t)j * d, valid, dist, gpos != nullptr, d, phi, g, lig, G);
+        const float sc = score_group(Kt + (size_t)j * d, valid, dist, gpos != nullptr, d, phi, g, lig, G, members);
         const float ss = a.flat_sig ? 1.f : sumsq_row(Vt + (size_t)j * d, valid, d, lig, G);
         if (valid && lig == 0) {
             if (a.scores) a.scores[(long long)id.e * N + j] = sc;
@@ -219,7 +260,7 @@ constexpr int kScoreRows = 64;  // rows per CTA
 template <typename T>
 __global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
     __shared__ unsigned long long phi[kMaxHalf];
-    __shared__ float2 g[kMaxHalf];
+    __shared__ float2 g[kMaxGroup * kMaxHalf];
     __shared__ int redi[kWarps];
     const DevLayout& lay = a.lay;
     const int row_blocks = (lay.N + kScoreRows - 1) / kScoreRows;
@@ -231,7 +272,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int* gpos = event_pos(a.pos, id);
     for (int f = tid; f < d / 2; f += kThreads) phi[f] = tab.phi[f];
-    fold_query(a.qstat + ((long long)id.l * lay.H + id.h) * d, tab, d, g);
+    const int members = fold_group(a, id, tab, d, g);
     long long pref = 0;
     if (gpos) {
         if (a.p_ref) pref = a.p_ref[id.b];
@@ -252,7 +293,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const EventArgs a, cons
         const bool valid = j < rend;
         const long long dist = (valid && gpos) ? pref - (long long)gpos[j] : 0;
         const T* krow = Kg + (valid ? row_offset(lay, id.b, id.l, id.h, j) : 0);
-        const float sc = score_row(krow, valid, dist, gpos != nullptr, d, phi, g, lig, G);
+        const float sc = score_group(krow, valid, dist, gpos != nullptr, d, phi, g, lig, G, members);
         if (valid && lig == 0) {
             a.scores[(long long)id.e * lay.N + j] = sc;
             bad |= !isfinite(sc);

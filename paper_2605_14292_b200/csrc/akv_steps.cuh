@@ -23,17 +23,6 @@ struct LayoutRows {
 };
 
 // ---- score ------------------------------------------------------------------------------------
-// Folded query statistic g_f = c_f * z(q)_f / sqrt(d) for f < d/2, written to shared memory.
-__device__ __forceinline__ void fold_query(const float* __restrict__ q, const ScoreTab& tab, int d, float2* g) {
-    const int half = d >> 1;
-    const float inv = rsqrtf((float)d);
-    for (int f = threadIdx.x; f < half; f += blockDim.x) {
-        const float qr = q[f] * inv, qi = q[f + half] * inv;
-        const float2 c = tab.cw[f];
-        g[f] = make_float2(c.x * qr - c.y * qi, c.x * qi + c.y * qr);
-    }
-}
-
 // cos and sin of 2*pi*(top / 2^32): octant reduction on the fixed-point phase, then short polynomials
 // in y = (angle offset)/(pi/4) in [-1, 1) (least-squares fits at Chebyshev nodes, |error| < 1e-7).
 __device__ __forceinline__ void sincos_phase(uint32_t top, float& sn, float& cs) {

@@ -76,6 +76,10 @@ extern "C" void akv_default_options(akv_options_t* o) {
     o->future_window = 1;
     o->sig_mode = AKV_SIG_PER_HEAD;
     o->flags = 0;
+    o->head_budgets = nullptr;
+    o->shared_gram = nullptr;
+    o->gqa_group = 1;
+    o->gqa_reduce = 0;
 }
 
 extern "C" akv_status_t akv_create(akv_handle_t** out, int device) {
@@ -182,6 +186,8 @@ static akv_status_t check_options(const akv_options_t* o) {
     if (!(o->eps >= 0.f) || !std::isfinite(o->eps)) return fail(AKV_ERR_INVALID_ARG, "eps must be finite and >= 0");
     if (!(o->rope_base > 0.f) || !std::isfinite(o->rope_base)) return fail(AKV_ERR_INVALID_ARG, "rope_base must be positive");
     if (o->future_window < 1 || o->future_window > 65536) return fail(AKV_ERR_INVALID_ARG, "future_window must be in 1..65536");
+    if (o->gqa_group < 0 || o->gqa_group > kMaxGroup) return fail(AKV_ERR_INVALID_ARG, "gqa_group must be in 0..%d", kMaxGroup);
+    if (o->gqa_reduce != 0 && o->gqa_reduce != 1) return fail(AKV_ERR_INVALID_ARG, "gqa_reduce must be 0 (mean) or 1 (max)");
     if (o->sig_mode != AKV_SIG_PER_HEAD && o->sig_mode != AKV_SIG_FLAT && o->sig_mode != AKV_SIG_PER_LAYER)
         return fail(AKV_ERR_UNSUPPORTED, "sig_mode %d", (int)o->sig_mode);
     return AKV_OK;
@@ -245,6 +251,11 @@ struct DeviceGuard {
     ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
+static void fill_score_args(EventArgs& a, const akv_options_t* opt) {
+    a.gqa_group = opt->gqa_group < 1 ? 1 : opt->gqa_group;
+    a.gqa_max = opt->gqa_reduce == 1 && a.gqa_group > 1;
+}
+
 // ------------------------------------------------------------------------------------------------
 // launch helpers
 // ------------------------------------------------------------------------------------------------
@@ -292,7 +303,7 @@ static akv_status_t launch_select_t(akv_handle* h, const EventArgs& a, cudaStrea
 
 // Tensor-memory path (bf16, d = 128, per-head signatures, N <= 256): one CTA of four warps per event.
 static bool tc_path_ok(const EventArgs& a) {
-    return a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.flat_sig == nullptr;
+    return a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.flat_sig == nullptr && a.gqa_group <= 1;
 }
 template <bool FUSED>
 static akv_status_t launch_tc(akv_handle* h, const EventArgs& a0, cudaStream_t st, bool dry = false) {
@@ -319,7 +330,7 @@ static bool tri_path_ok(const EventArgs& a) { return tc_path_ok(a) && (a.lay.N <
 static bool tri_big_ok(const EventArgs& a) { return tc_path_ok(a) && !tri_path_ok(a) && a.budget <= 128; }
 // shared signatures with their cosine matrix at hand: the large size, which gathers its triangle from that matrix
 static bool pool_shared_ok(const EventArgs& a) {
-    return a.gram != nullptr && a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.budget <= 128;
+    return a.gram != nullptr && a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N <= kTcMaxN && a.budget <= 128 && a.gqa_group <= 1;
 }
 template <bool FUSED, bool BIG>
 static akv_status_t launch_tri(akv_handle* h, const EventArgs& a, cudaStream_t st, bool dry = false) {
@@ -395,6 +406,7 @@ static akv_status_t alpha_score_impl(akv_handle_t* h, const akv_layout_t* lay, c
     a.pos = PosDesc{const_cast<int*>(pos), psb, psl, psh};
     a.n_cand = n_cand; a.qstat = qstat; a.p_ref = p_ref;
     a.scores = scores; a.status = status;
+    fill_score_args(a, opt);
     return launch_score(h, a, (cudaStream_t)stream);
 }
 
@@ -504,7 +516,7 @@ enum EventRoute { ROUTE_TRI, ROUTE_TRI_BIG, ROUTE_TC, ROUTE_STREAM, ROUTE_RESIDE
 // shared memory the streaming kernel may plan with: what the device allows minus its static arrays
 static int stream_smem_limit(int smem_optin) { return smem_optin - 1024; }
 static bool stream_path_ok(const EventArgs& a, int smem_optin) {
-    if (!(a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N > kTcMaxN && a.lay.N <= 65535 && a.flat_sig == nullptr)) return false;
+    if (!(a.lay.dtype == AKV_BF16 && a.lay.d == kTcD && a.lay.N > kTcMaxN && a.lay.N <= 65535 && a.flat_sig == nullptr && a.gqa_group <= 1)) return false;
     const StSmem sp = plan_st_smem(a.lay.N, a.budget, stream_smem_limit(smem_optin));
     return sp.cap_rows > 0 && (int)sp.total <= stream_smem_limit(smem_optin);
 }
@@ -533,6 +545,7 @@ extern "C" akv_status_t akv_workspace_bytes(const akv_layout_t* lay, int32_t bud
     // only whether shared signatures are in use matters for the route, not where they live
     a.flat_sig = opt->sig_mode != AKV_SIG_PER_HEAD ? reinterpret_cast<const float*>(bytes) : nullptr;
     a.gram = opt->sig_mode != AKV_SIG_PER_HEAD ? opt->shared_gram : nullptr;
+    fill_score_args(a, opt);
     int dev = 0, smem_optin = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     CUDA_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
@@ -573,6 +586,7 @@ static akv_status_t alpha_compress_event_impl(akv_handle_t* h, const akv_layout_
     if (!aligned16(K) || !aligned16(V)) return fail(AKV_ERR_ALIGNMENT, "alpha_compress_event: K/V must be 16-byte aligned");
     if ((s = check_pos_written(a.lay, pos, psb, psl, psh)) != AKV_OK) return s;
     if ((s = fill_select_args(a, opt, V, flat_sig)) != AKV_OK) return s;
+    fill_score_args(a, opt);
     DeviceGuard guard(h->device);
     if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
     build_tables(h, lay->d, opt->rope_base, opt->future_window);
@@ -668,6 +682,7 @@ static akv_status_t alpha_compress_event_static_impl(akv_handle_t* h, const akv_
     if ((s = fill_select_args(a, opt, V, flat_sig)) != AKV_OK) return s;
     DeviceGuard guard(h->device);
     if (!guard.ok) return fail(AKV_ERR_CUDA, "cannot select device %d", h->device);
+    fill_score_args(a, opt);
     float* scratch = nullptr;
     if ((s = static_scores_address(h->device, &scratch)) != AKV_OK) return s;
     build_tables(h, lay->d, opt->rope_base, opt->future_window);

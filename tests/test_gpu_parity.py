@@ -559,6 +559,36 @@ def test_fused_event_with_shared_cosine_matrix(mode, N, budget):
     assert int(sel.status.abs().max()) == 0 and int(sel.n_kept.min()) == budget
 
 
+# ------------------------------------------------------------------ grouped-query statistics
+@pytest.mark.parametrize("reduce", ["mean", "max"])
+@pytest.mark.parametrize("dtype,N,d", [(synth.BF16, 150, 128), (synth.F32, 600, 64)])
+def test_grouped_query_statistics(reduce, dtype, N, d):
+    """Several query statistics per KV head: scores are the mean or the maximum over the group (stand-alone scorer),
+    and the fused call selects with them (resident kernel for the small shape, three launches for the large one)."""
+    G = 4
+    ev = synth.make_plain(2, 2, 2, N, d, 30, 0.5, dtype=dtype, seed=101)
+    rng = np.random.default_rng(102)
+    Q = rng.standard_normal((2, 2 * G, d)).astype(np.float32)            # [L, H * G, d]
+    K, V, pos, pref = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.p_ref)
+    opts = akv.Options(lam=0.5, gqa_group=G, gqa_reduce=akv.GQA_MAX if reduce == "max" else akv.GQA_MEAN)
+    s = akv.alpha_score(K, dev(Q), pos=pos, p_ref=pref, opts=opts).cpu().numpy()
+    sel = akv.alpha_compress_event(K, V, pos, dev(Q), 30, opts, p_ref=pref, want_scores=True)
+    torch.cuda.synchronize()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    for b in range(2):
+        for l in range(2):
+            for h in range(2):
+                qs = Q[l, h * G:(h + 1) * G]
+                ref = O.triattention_score_group(ev.K[b, l, h], ev.pos[b, l, h], qs, int(ev.p_ref[b]), reduce=reduce)
+                scale = max(chk.score_scale(ev.K[b, l, h], q, d).max() for q in qs) * np.ones(N)
+                chk.check_scores(s[b, l, h], ref, scale)
+                chk.check_event(ev.K[b, l, h], ev.V[b, l, h], ev.pos[b, l, h], qs[0], int(ev.p_ref[b]), 30, 0.5,
+                                None, sel.pick_order[b, l, h].cpu().numpy(), sel.idx_sorted[b, l, h].cpu().numpy(),
+                                Kn[b, l, h], Vn[b, l, h], pn[b, l, h], ref_scores=ref)
+                assert np.max(np.abs(sel.scores[b, l, h].cpu().numpy() - ref)) < 1e-5 * scale.max()
+
+
+
 def test_report_worst_score_error():
     """Printed for the record (run last in this file): the worst score error of everything checked so far."""
     print("worst |err|/|s| where |s| >= 0.1 scale: %.3e; worst |err|/scale: %.3e; scores checked: %d"

@@ -152,3 +152,23 @@ def test_bf16_round_trip_and_rounding():
     assert back[3] == np.float32(-2.5)
     assert abs(back[4] - 3.140625) < 1e-7
     assert np.array_equal(O.widen(bits), back.astype(np.float64))
+
+
+def test_group_score_reduces_to_the_plain_score_and_to_linearity():
+    """Grouped queries: one member is the plain score; the mean over members is the score of the mean statistic
+    (the score is linear in it); the maximum is reached by a member at every key and does not depend on the
+    members' order."""
+    rng = np.random.default_rng(20)
+    n, d, G = 23, 16, 4
+    K = rng.standard_normal((n, d)).astype(np.float32)
+    Q = rng.standard_normal((G, d)).astype(np.float32)
+    pos = np.sort(rng.choice(500, size=n, replace=False))
+    one = O.triattention_score_group(K, pos, Q[:1], 600, 2)
+    assert np.array_equal(one, O.triattention_score(K, pos, Q[0], 600, 2))
+    mean = O.triattention_score_group(K, pos, Q, 600, 2, reduce="mean")
+    assert np.max(np.abs(mean - O.triattention_score(K, pos, Q.astype(np.float64).mean(axis=0), 600, 2))) < 1e-12
+    mx = O.triattention_score_group(K, pos, Q, 600, 2, reduce="max")
+    each = np.stack([O.triattention_score(K, pos, q, 600, 2) for q in Q])
+    assert np.all(mx >= each - 0) and np.all(np.isin(mx, each))
+    assert np.array_equal(mx, O.triattention_score_group(K, pos, Q[::-1], 600, 2, reduce="max"))
+    assert np.all(mx >= mean - 1e-12)

@@ -511,6 +511,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                     if (32 * cb + k < nb) tri[tri_row(128 + 32 * cb + k) + rho] = __uint_as_float(v[k]);
             }
             const int ra = base2 + rho - 128;  // this thread's row of the second product, counted from row 128
+            float diag = 0.f;                  // its squared norm (one square root and one division per thread, after the loop)
             for (int cb = 0; cb < (nb + 31) >> 5; ++cb) {
                 uint32_t v[32];
                 tmem_ld32(lanes + (uint32_t)ncols + (uint32_t)(32 * cb), v);
@@ -519,10 +520,11 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
 #pragma unroll
                     for (int k = 0; k < 32; ++k) {
                         if (32 * cb + k <= ra) tri[tri_row(128 + ra) + 128 + 32 * cb + k] = __uint_as_float(v[k]);
-                        if (32 * cb + k == ra) r[128 + ra] = 1.f / (sqrtf(__uint_as_float(v[k])) + a.eps);
+                        diag = (32 * cb + k == ra) ? __uint_as_float(v[k]) : diag;
                     }
                 }
             }
+            if (ra >= 0 && ra < nb) r[128 + ra] = 1.f / (sqrtf(diag) + a.eps);
         }
     } else if (slow) {
         // reciprocal norms (Eq. 1); this pool does not fit the tile, its V rows are read in place

@@ -484,6 +484,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
                 if (128 * blk + 32 * (warp & 3) < R) {
                     const uint32_t lanes = tbase + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(256 * blk);
                     const int trow = tri_row(row), last_cb = (128 * blk + 32 * (warp & 3) + 31) >> 5;
+                    float diag = 0.f;  // the diagonal entry: squared norm
                     for (int cb = 0; cb <= last_cb; ++cb) {
                         uint32_t v[32];
                         tmem_ld32(lanes + (uint32_t)(32 * cb), v);
@@ -492,10 +493,11 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
 #pragma unroll
                             for (int k = 0; k < 32; ++k) {
                                 if (32 * cb + k <= row) tri[trow + 32 * cb + k] = __uint_as_float(v[k]);
-                                if (32 * cb + k == row) ar[row] = 1.f / (sqrtf(__uint_as_float(v[k])) + a.eps);  // the diagonal: squared norm
+                                diag = (32 * cb + k == row) ? __uint_as_float(v[k]) : diag;
                             }
                         }
                     }
+                    if (row < R) ar[row] = 1.f / (sqrtf(diag) + a.eps);
                 }
             }
             tc_fence_before();
@@ -822,10 +824,8 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
 
     phase_stamp(id.e, 6);
     // ---- sort(S) and outputs -------------------------------------------------------------------------
-    {
-        const int kept = ordered_scan([&](int j) { return taken[j] != 0; }, [&](int j, int pos) { idx[pos] = j; });
-        for (int t = kept + tid; t < a.budget; t += kStWork) idx[t] = -1;
-    }
+    const int kept = ordered_scan([&](int j) { return taken[j] != 0; }, [&](int j, int pos) { idx[pos] = j; });
+    for (int t = kept + tid; t < a.budget; t += kStWork) idx[t] = -1;
     work_barrier();
     const long long ob = (long long)id.e * a.budget;
     for (int t = tid; t < a.budget; t += kStWork) {
@@ -844,8 +844,9 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     // and idx[t] >= t; later chunks' sources lie at or beyond their own destinations)
     int* wpos = a.pos.p ? a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh : nullptr;
     const int chunk = (int)(kStStageChunk / 512u);  // rows of K and of V staged per round
-    for (int c0 = 0; c0 < picks; c0 += chunk) {
-        const int cn = min(chunk, picks - c0);
+    const int moved = min(picks, kept);  // (equal by construction; the smaller one keeps every index read below valid)
+    for (int c0 = 0; c0 < moved; c0 += chunk) {
+        const int cn = min(chunk, moved - c0);
         work_barrier();
         for (int x = tid; x < cn * 16; x += kStWork) {
             const long long off = rowoff(idx[c0 + (x >> 4)]) + (x & 15) * 8;

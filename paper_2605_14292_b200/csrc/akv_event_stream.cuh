@@ -509,7 +509,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
             }
             phase_stamp(id.e, 5);
             if (warp == 0) {
-                const bool ok = picks_bounded<8, true>(lane, R, picks, true, s, act, ar, a.lam, reinterpret_cast<const float*>(tile),
+                const bool ok = picks_cosine<8, true>(lane, R, picks, s, act, ar, a.lam, reinterpret_cast<float*>(tile),
                                                            reinterpret_cast<uint32_t*>(gain), order, bound);
                 if (lane == 0) cnt[2] = ok ? 1 : 0;
             }

@@ -4,8 +4,8 @@
 // memory, Algorithm 1 as a one-warp loop), for an ACTIVE SET instead of the whole pool:
 //
 //   The picks hardly ever reach beyond the best-scored few dozen rows past the budget. The cosine matrix is
-//   therefore formed only for the pool's best-scored rows, at most 176 of them (61 KB of triangle: three CTAs
-//   per SM), and only their V rows are read. Every candidate left out scores at most `bound`, the 177th largest
+//   therefore formed only for the pool's best-scored rows, at most 180 of them (64 KB of triangle: three CTAs
+//   per SM), and only their V rows are read. Every candidate left out scores at most `bound`, the 181st largest
 //   key, and its Eq. 2 value never exceeds its score: the loop over the active set is exact as long as its
 //   winning value stays above that bound. In the rare event where it does not, the event is redone over its whole
 //   pool with rows of the cosine matrix taken as plain dot products.
@@ -19,11 +19,12 @@ namespace akv {
 
 // Two sizes of the kernel. The small one (budgets up to 64): a tile of 128 rows of 256 bytes, which holds the V
 // operand and then the triangle of a pool of up to 127 rows; six CTAs per SM. The large one (budgets up to 128,
-// N up to 256): 61 KB, for the triangle of an active set of up to 176 rows (see the kernel); three CTAs per SM.
+// N up to 256): 64 KB, for a whole event's K rows, then the triangle of an active set of up to 180 rows (see the kernel); three CTAs per SM.
 template <bool BIG>
 struct TriCfg {
-    static constexpr unsigned kTileBytes = BIG ? 62464u : 32768u;
-    static constexpr int kMaxPool = BIG ? 176 : 127;     // most rows whose cosine matrix goes through the tile
+    static constexpr unsigned kTileBytes = BIG ? 65536u : 32768u;
+    static constexpr int kKRows = BIG ? 256 : 128;       // K rows resident at a time (the large tile holds a whole event)
+    static constexpr int kMaxPool = BIG ? 180 : 127;     // most rows whose cosine matrix goes through the tile
     static constexpr uint32_t kCols = BIG ? 256u : 128u;  // tensor-memory columns (a power of two >= the matrix's columns)
     static constexpr int kCpl = BIG ? 6 : 4;             // candidates per lane of the one-warp loop
 };
@@ -115,9 +116,8 @@ constexpr float kLowestScore = -3.0e38f;
 // The loop of Algorithm 1 with the cosine penalty, Eq. 2 evaluated and compared as floats (no integer keys):
 // a candidate is retired through the triangle itself. The diagonal entries are set to +inf before the first
 // pick, so the update m <- max(m, Sims[i, :]) gives the picked row m = +inf and a = -inf from then on: no
-// mask, no per-candidate retirement. Each lane keeps the best of its candidates and which one it is while it
-// evaluates them (a compare tree), so the second reduction's operand costs three instructions per pick, not
-// three per candidate. Winning values are parked as order-preserving keys, like the other loops'.
+// mask, no per-candidate retirement. Each lane reduces its candidates to one maximum before the warp-wide
+// reduction and finds which candidate that was while the reduction is in flight. Winning values are parked as order-preserving keys, like the other loops'.
 // BOUNDED as for picks_bounded. `tri` is modified (its diagonal).
 template <int CPL, bool BOUNDED>
 __device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const float* s, const unsigned short* bypool,
@@ -150,13 +150,17 @@ __device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const f
         const int t1 = min(t0 + 32, picks);
         for (int t = t0; t < t1; ++t) {
             float bv[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) bv[k] = fmaf(-lr[k], M[k], sv[k]);
+            float lm = bv[0];
+#pragma unroll
+            for (int k = 1; k < CPL; ++k) lm = fmaxf(lm, bv[k]);
+            const float whi = warp_max_f32(lm);
+            // which of the lane's candidates that was, the lower row on equal values (a compare tree, independent of
+            // the reduction in flight)
             int bi[CPL];
 #pragma unroll
-            for (int k = 0; k < CPL; ++k) {
-                bv[k] = fmaf(-lr[k], M[k], sv[k]);
-                bi[k] = lane + 32 * k;
-            }
-            // best of the lane's candidates, the lower row on equal values
+            for (int k = 0; k < CPL; ++k) bi[k] = lane + 32 * k;
 #pragma unroll
             for (int w = 1; w < CPL; w *= 2) {
 #pragma unroll
@@ -166,8 +170,8 @@ __device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const f
                     bi[k] = gt ? bi[k + w] : bi[k];
                 }
             }
-            const float whi = warp_max_f32(bv[0]);
-            const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, bv[0] == whi ? 0xFFFFu - (uint32_t)bi[0] : 0u);
+            const int row = bi[0];
+            const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, lm == whi ? 0xFFFFu - (uint32_t)row : 0u);
             const int irho = min((int)(0xFFFFu - wlo), last);
             if (BOUNDED && whi <= bound) return false;
             const bool mine = lane == t - t0;
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             row += run;
         }
     };
-    const int n_late = FUSED && n > kTriTileRows ? n - kTriTileRows : 0;  // rows that wait for a free slot
+    const int n_late = FUSED && n > Cfg::kKRows ? n - Cfg::kKRows : 0;  // rows that wait for a free slot
     if (tid == 0) {
         mbar_init(barK, 1);
         mbar_init(barM, 1);
@@ -338,7 +342,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                 }
                 float acc = 0.f;
                 if (live) {
-                    const unsigned char* krow = tile + (j & (kTriTileRows - 1)) * 256 + (lane & 7) * 16;
+                    const unsigned char* krow = tile + (j & (Cfg::kKRows - 1)) * 256 + (lane & 7) * 16;
                     acc = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
                 }
 #pragma unroll
@@ -358,13 +362,13 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         for (int pass = 0; pass < 2; ++pass) {
             // first and third stretch share one copy of the loop (the kernel's code should stay small)
             if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0, a.wait_polls);
-            score_rounds(pass ? kTriTileRows / 16 : 0, pass ? rounds : late_round);
+            score_rounds(pass ? Cfg::kKRows / 16 : 0, pass ? rounds : late_round);
             if (!pass) {
                 if (n_late > 0) {
                     __syncthreads();
-                    if (tid == 0) request_k_rows(kTriTileRows, n, 0, barL);
+                    if (tid == 0) request_k_rows(Cfg::kKRows, n, 0, barL);
                 }
-                score_rounds(late_round, min(rounds, kTriTileRows / 16));
+                score_rounds(late_round, min(rounds, Cfg::kKRows / 16));
             }
         }
     } else {
@@ -782,6 +786,21 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             const unsigned char* src = tile + slot0 + (t - r0) * 256;
             *reinterpret_cast<uint4*>(Kg + off) = *reinterpret_cast<const uint4*>(src);
             *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(src + 16384);
+        }
+    } else if ((unsigned)picks * 512u <= Cfg::kTileBytes) {
+        // the tile holds the kept rows of K and of V side by side: one round of loads, one barrier, one of stores
+        const uint32_t vhalf = Cfg::kTileBytes / 2u;
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
+            cp_async16(tile_u32 + (uint32_t)x * 16u, Kg + off);
+            cp_async16(tile_u32 + vhalf + (uint32_t)x * 16u, Vg + off);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        for (int x = tid; x < picks * 16; x += kTcThreads) {
+            const long long off = rowoff(x >> 4) + (x & 15) * 8;
+            copy16(reinterpret_cast<char*>(Kg + off), tile + x * 16);
+            copy16(reinterpret_cast<char*>(Vg + off), tile + vhalf + x * 16);
         }
     } else {
 #pragma unroll 1

@@ -322,6 +322,14 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         const long long D16 = n > 16 ? (long long)spos[n - 1] - (long long)spos[n - 17] : 0;
         ChainScore cs;
         cs.set_step(D16, phitab + f0, sect);
+        // whether every row sits D16 after the row 16 slots before it (found once; the chains then need no look at
+        // the positions)
+        bool uniform = false;
+        if (BIG) {
+            bool uni = true;
+            for (int j = 16 + tid; j < n; j += kTcThreads) uni &= (long long)spos[j] - (long long)spos[j - 16] == D16;
+            uniform = __syncthreads_and(uni);
+        }
         const int rounds = (n + 15) >> 4, late_round = (n_late + 15) >> 4;
         // 16 rows per round (4 per warp), in three stretches. Rows from 128 on reuse the slots of rows
         // 0..n_late-1: they are requested after the first stretch, once every warp is past those rows,
@@ -358,8 +366,72 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             }
         };
         timeout = !mbar_wait_bounded(barK, 0, a.wait_polls);
+        phase_stamp(id.e, 10);  // (K rows have arrived)
+        if (BIG) {
+            // The tile holds the whole event. A lane group scores two rows side by side, row j of the first half
+            // of the rounds and row j + 16 * half of the second: two independent chains that share the turn S, so
+            // that one chain's dependent arithmetic fills the other's latency.
+            const int half = (rounds + 1) >> 1;
+            ChainScore cb;
+            AKV_PHASE_ACC_DECL(cyc_anchor);
 #pragma unroll 1
-        for (int pass = 0; pass < 2; ++pass) {
+            for (int round = 0; round < half; ++round) {
+                const int ja = 16 * round + 4 * warp + grp, jb = ja + 16 * half;
+                const bool la = ja < n, lb = jb < n;
+                // each chain on its own: after an event the kept rows' positions are irregular (fresh rotation every
+                // round) while the rows appended since are consecutive (chained)
+                bool fa = round == 0 || a.no_chain, fb = fa;
+                if (!fa && !uniform) {
+                    fa = !__all_sync(0xFFFFFFFFu, !la || (long long)spos[ja] - (long long)spos[ja - 16] == D16);
+                    fb = !__all_sync(0xFFFFFFFFu, !lb || (long long)spos[jb] - (long long)spos[jb - 16] == D16);
+                }
+                AKV_PHASE_ACC_BEGIN(cyc_anchor);
+                if (fa) {
+                    if (la) cs.anchor(pref - (long long)spos[ja], gtab + f0, phitab + f0, sect);
+                } else {
+                    cs.advance();
+                }
+                if (fb) {
+                    if (lb) cb.anchor(pref - (long long)spos[jb], gtab + f0, phitab + f0, sect);
+                } else {
+                    cb.advance_by(cs);
+                }
+                AKV_PHASE_ACC_END(cyc_anchor);
+                float acca = 0.f, accb = 0.f;
+                if (la) {
+                    const unsigned char* krow = tile + ja * 256 + (lane & 7) * 16;
+                    acca = cs.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
+                }
+                if (lb) {
+                    const unsigned char* krow = tile + jb * 256 + (lane & 7) * 16;
+                    accb = cb.dot(*reinterpret_cast<const uint4*>(krow), *reinterpret_cast<const uint4*>(krow + 128));
+                }
+#pragma unroll
+                for (int off = 4; off > 0; off >>= 1) {
+                    acca += __shfl_xor_sync(0xFFFFFFFFu, acca, off);
+                    accb += __shfl_xor_sync(0xFFFFFFFFu, accb, off);
+                }
+                if ((lane & 7) == 0) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int j = h ? jb : ja;
+                        const float acc = h ? accb : acca;
+                        if (j < n) {
+                            if (a.scores) a.scores[(long long)id.e * N + j] = acc;
+                            const bool fin = isfinite(acc);
+                            bad |= !fin;
+                            const float sj = fin ? acc : -INFINITY;
+                            s[j] = sj;
+                            key[j] = orderable(sj);
+                        }
+                    }
+                }
+            }
+            AKV_PHASE_ACC_STORE(id.e, 11, cyc_anchor);
+            phase_stamp(id.e, 12);  // (scoring loop left)
+        }
+#pragma unroll 1
+        for (int pass = 0; !BIG && pass < 2; ++pass) {
             // first and third stretch share one copy of the loop (the kernel's code should stay small)
             if (pass && n_late > 0) timeout |= !mbar_wait_bounded(barL, 0, a.wait_polls);
             score_rounds(pass ? Cfg::kKRows / 16 : 0, pass ? rounds : late_round);

@@ -176,6 +176,15 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     __syncthreads();
     long long pref = 0;
     if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)cnt[1] + 1;
+    // D: the spacing of rows one stage (64 slots) apart at the newest end, which a cache filled token by token has
+    // everywhere. Whether it does is found once, here; the scoring loop then chains without looking at positions.
+    const long long D = n > kStStageRows ? (long long)spos[n - 1] - (long long)spos[n - 1 - kStStageRows] : 0;
+    bool uniform;
+    {
+        bool uni = true;
+        for (int j = kStStageRows + tid; j < n; j += kStThreads) uni &= (long long)spos[j] - (long long)spos[j - kStStageRows] == D;
+        uniform = __syncthreads_and(uni);
+    }
 
     phase_stamp(id.e, 1);
     // ---- K through the ring, scored as it lands ---------------------------------------------------------------
@@ -206,9 +215,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     } else {
         const int grp = lane >> 3, f0 = (lane & 7) * 8;
         // A lane group scores two rows of every stage, 32 slots apart, as two independent chains (the second
-        // hides the first one's latencies); each chain steps by one stage = 64 slots. D: the spacing of rows 64
-        // slots apart at the newest end, which a cache filled token by token has everywhere.
-        const long long D = n > kStStageRows ? (long long)spos[n - 1] - (long long)spos[n - 1 - kStStageRows] : 0;
+        // hides the first one's latencies); each chain steps by one stage = 64 slots.
         const int D32 = (int)D;
         const bool d_fits = (long long)D32 == D;
         ChainScore ca, cb;  // cb uses ca's S
@@ -221,9 +228,13 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
             }
             const int ja = st * kStStageRows + 4 * warp + grp, jb = ja + kStRoundRows;
             const bool la = ja < n, lb = jb < n;
-            const int pa = la ? spos[ja] : 0, pb = lb ? spos[jb] : 0;
             bool fresh = (st & (kChainRounds - 1)) == 0 || a.no_chain || !d_fits;
-            if (!fresh)
+            int pa = 0, pb = 0;
+            if (fresh || !uniform) {
+                pa = la ? spos[ja] : 0;
+                pb = lb ? spos[jb] : 0;
+            }
+            if (!fresh && !uniform)
                 fresh = !__all_sync(0xFFFFFFFFu, (!la || pa - spos[ja - kStStageRows] == D32) && (!lb || pb - spos[jb - kStStageRows] == D32));
             if (fresh) {
                 if (la) ca.anchor(pref - (long long)pa, gtab + f0, phitab + f0, sect);

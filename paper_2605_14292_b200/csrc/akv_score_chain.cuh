@@ -80,6 +80,18 @@ struct ChainScore {
         }
         return acc2.x + acc2.y;
     }
+    // the same sum with four independent accumulators (a chain of two dependent products instead of eight)
+    __device__ __forceinline__ float dot4(const uint4& wr, const uint4& wi) const {
+        const uint32_t wre[4] = {wr.x, wr.y, wr.z, wr.w}, wim[4] = {wi.x, wi.y, wi.z, wi.w};
+        float2 acc[4];
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+            acc[p] = __ffma2_rn(Gy[p], make_float2(bf16lo(wim[p]), bf16hi(wim[p])),
+                                __fmul2_rn(Gx[p], make_float2(bf16lo(wre[p]), bf16hi(wre[p]))));
+        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+        const float2 a = __fadd2_rn(a01, a23);
+        return a.x + a.y;
+    }
 };
 constexpr int kChainRounds = 8;        // rounds between two fresh computations of G (long events, streamed)
 constexpr int kChainRoundsShort = 16;  // the same for events of at most 256 rows: one or two fresh computations per lane

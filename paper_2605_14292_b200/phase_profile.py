@@ -20,6 +20,8 @@ from . import api, build, synth
 PHASES = {
     "event_tri_kernel": ["tensor memory claimed", "K scored", "s_(b) + pool", "V operand", "product", "triangle",
                          "picks (one warp)", "sort + outputs", "compaction"],
+    "event_pool_kernel": ["tensor memory claimed", "K scored", "s_(b) + pool", "V operand", "product", "triangle",
+                          "picks (one warp)", "sort + outputs", "compaction"],
     "event_tc_kernel": ["K scored", "ranks + pool", "V operand + tensor memory", "product + norms", "picks",
                         "sort + outputs", "compaction"],
     "event_stream_kernel": ["tables + positions", "K streamed and scored", "s_(b)", "pool / top-k", "V rows + norms",
@@ -40,7 +42,7 @@ def main():
     slots = int(lib.akv_debug_phase_slots())
     dev = torch.device("cuda")
     if args.config == "C2":
-        ev, kernel = synth.make_c2(B=args.batch or 1), "event_tri_kernel"
+        ev, kernel = synth.make_c2(B=args.batch or 1), "event_pool_kernel"
     elif args.config == "C3":
         ev, kernel = synth.make_c3(B=args.batch or 16), "event_tri_kernel"
     elif args.config == "C4":
@@ -51,7 +53,7 @@ def main():
         V = synth.paged_gather_dense(c5.pool_V, c5.block_table)
         ev = synth.EventBatch("C5-round0", synth.BF16, K, V, c5.pos, c5.qstat, np.full((c5.B,), 256, dtype=np.int32),
                               c5.budget, c5.lam)
-        kernel = "event_tri_kernel"
+        kernel = "event_pool_kernel"
     K, V, pos = api.to_device(ev.K, dev), api.to_device(ev.V, dev), api.to_device(ev.pos, dev)
     q, pref = api.to_device(ev.qstat, dev), api.to_device(ev.p_ref, dev)
     E = ev.n_events
@@ -80,6 +82,14 @@ def main():
     if kernel == "event_stream_kernel" and np.any(st[:, 10] > 0):
         for k, name in ((10, "  of picks: arg-max + exchange"), (11, "  of picks: products (misses)"), (12, "  of picks: tensor-memory read")):
             print(f"  {name:32s} {np.median(st[:, k]):10.0f} {st[:, k].mean():10.0f}")
+    if kernel == "event_pool_kernel" and np.any(st[:, 10] > 0):
+        ok = (st[:, 10] > 0) & (st[:, 1] > 0)
+        d = (st[ok, 10] - st[ok, 1]).astype(np.float64)
+        print(f"  {'  of K scored: until K arrived':32s} {np.median(d):10.0f} {d.mean():10.0f}")
+        if np.any(st[:, 12] > 0):
+            d = (st[ok, 12] - st[ok, 10]).astype(np.float64)
+            print(f"  {'  of K scored: scoring loop':32s} {np.median(d):10.0f} {d.mean():10.0f}")
+            print(f"  {'    of which rotations (fresh or chained)':32s} {np.median(st[ok, 11]):10.0f} {st[ok, 11].mean():10.0f}")
     life = (st[:, len(names)] - st[:, 0]).astype(np.float64)
     life = life[(st[:, len(names)] > 0) & (st[:, 0] > 0)]
     print(f"  {'CTA lifetime':32s} {np.median(life):10.0f} {life.mean():10.0f}")

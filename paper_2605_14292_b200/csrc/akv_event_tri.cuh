@@ -178,6 +178,102 @@ __device__ __forceinline__ void picks_in_one_warp(int lane, int P, int picks, bo
     }
 }
 
+// Warp-wide maximum of a float (sm_100a has the reduction for f32).
+__device__ __forceinline__ float warp_max_f32(float v) {
+    float m;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
+    return m;
+}
+
+// A non-finite score competes as this value: below every real score, above a retired candidate's -inf.
+constexpr float kLowestScore = -3.0e38f;
+
+// The loop of Algorithm 1 with the cosine penalty, Eq. 2 evaluated and compared as floats (no integer keys):
+// a candidate is retired through the triangle itself. The diagonal entries are set to +inf before the first
+// pick, so the update m <- max(m, Sims[i, :]) gives the picked row m = +inf and a = -inf from then on: no
+// mask, no per-candidate retirement. Each lane reduces its candidates to one maximum before the warp-wide
+// reduction and finds which candidate that was while the reduction is in flight. Winning values are parked as order-preserving keys, like the other loops'.
+// BOUNDED as for picks_bounded. `tri` is modified (its diagonal).
+template <int CPL, bool BOUNDED>
+__device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const float* s, const unsigned short* bypool,
+                                             const float* r, float lam, float* tri, uint32_t* park_key, int* park_row,
+                                             uint32_t bound_key = 0u) {
+    const uint32_t tb = smem_u32(tri), rb = smem_u32(r);
+    const float ninf = __int_as_float(0xff800000), pinf = __int_as_float(0x7f800000);
+    float sv[CPL], lr[CPL], M[CPL];
+    int rc4[CPL];
+    uint32_t trowB[CPL];  // 4 * row, and the shared-memory address of that row of the triangle
+    const int last = max(P - 1, 0);
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) {
+        const int rho = lane + 32 * k;
+        const bool in = rho < P;
+        // rows beyond the pool: -inf from the start, and a positive factor so that -inf - lr * m stays -inf
+        sv[k] = in ? fmaxf(s[bypool[min(rho, last)]], kLowestScore) : ninf;
+        lr[k] = in ? fmaxf(lam * r[rho], 1e-30f) : 1.f;
+        M[k] = 0.f;
+        const int rc = min(rho, last);  // clamped: the loads stay inside the triangle, the loop needs no branch
+        rc4[k] = 4 * rc;
+        trowB[k] = tb + 4u * (uint32_t)tri_row(rc);
+        if (in) tri[tri_row(rho) + rho] = pinf;
+    }
+    __syncwarp();
+    const float bound = from_orderable(bound_key);
+    for (int t0 = 0; t0 < picks; t0 += 32) {
+        float my_val = 0.f;
+        int my_row = 0;
+        const int t1 = min(t0 + 32, picks);
+        for (int t = t0; t < t1; ++t) {
+            float bv[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) bv[k] = fmaf(-lr[k], M[k], sv[k]);
+            float lm = bv[0];
+#pragma unroll
+            for (int k = 1; k < CPL; ++k) lm = fmaxf(lm, bv[k]);
+            const float whi = warp_max_f32(lm);
+            // which of the lane's candidates that was, the lower row on equal values (a compare tree, independent of
+            // the reduction in flight)
+            int bi[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) bi[k] = lane + 32 * k;
+#pragma unroll
+            for (int w = 1; w < CPL; w *= 2) {
+#pragma unroll
+                for (int k = 0; k + w < CPL; k += 2 * w) {
+                    const bool gt = bv[k + w] > bv[k];
+                    bv[k] = gt ? bv[k + w] : bv[k];
+                    bi[k] = gt ? bi[k + w] : bi[k];
+                }
+            }
+            const int row = bi[0];
+            const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, lm == whi ? 0xFFFFu - (uint32_t)row : 0u);
+            const int irho = min((int)(0xFFFFu - wlo), last);
+            if (BOUNDED && whi <= bound) return false;
+            const bool mine = lane == t - t0;
+            my_val = mine ? whi : my_val;
+            my_row = mine ? irho : my_row;
+            if (t + 1 == picks) continue;
+            // m <- max(m, Sims[i, :]) from the triangle: entry (max, min); the picked row meets its diagonal
+            const int irho4 = 4 * irho;
+            const uint32_t tiB = tb + 4u * (uint32_t)tri_row(irho);
+            uint32_t addr[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) addr[k] = rc4[k] > irho4 ? trowB[k] + (uint32_t)irho4 : tiB + (uint32_t)rc4[k];
+            const float ri = fmaxf(lds_in_order(rb + (uint32_t)irho4), 1e-30f);
+            float x[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) x[k] = lds_in_order(addr[k]);
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) M[k] = fmaxf(M[k], ri * x[k]);
+        }
+        if (t0 + lane < picks) {
+            park_key[t0 + lane] = orderable(my_val <= -2.9e38f ? ninf : my_val);
+            park_row[t0 + lane] = my_row;
+        }
+    }
+    return true;
+}
+
 // FUSED: score + select + compact; otherwise selection only (scores are read from a.scores and
 // nothing is rewritten).
 template <bool FUSED>
@@ -520,7 +616,8 @@ __global__ void __launch_bounds__(kTcThreads) event_tri_kernel(const EventArgs a
     uint32_t* park_key = reinterpret_cast<uint32_t*>(gain);
     if (!slow) {
         if (warp == 0) {
-            if (P <= 128) picks_in_one_warp<4>(lane, P, picks, fast, s, bypool, r, a.lam, tri, park_key, order);
+            if (fast) picks_cosine<4, false>(lane, P, picks, s, bypool, r, a.lam, tri, park_key, order);
+            else if (P <= 128) picks_in_one_warp<4>(lane, P, picks, false, s, bypool, r, a.lam, tri, park_key, order);
             else picks_in_one_warp<8>(lane, P, picks, false, s, bypool, r, a.lam, tri, park_key, order);
         }
     } else {

@@ -51,6 +51,16 @@ __host__ __device__ inline TriSmem plan_tri_smem(int N, int budget, bool big) {
     return p;
 }
 
+// Shared memory -> global memory as one bulk copy (16-byte aligned, a multiple of 16 bytes), and the wait that
+// must precede leaving the CTA or reusing the source: until the copies issued by this thread have read it.
+__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
 // BOUNDED: the P rows are only the best-scored part of the pool, and every candidate left out scores at most
 // `bound_key` (as an order-preserving key), so its Eq. 2 value can never exceed that. The loop is exact as long
 // as the winning value stays above the bound; at the first pick that does not, it stops and returns false.
@@ -180,6 +190,8 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         mbar_init(barM, 1);
         mbar_init(barL, 1);
         mbar_init_fence();
+        // the K rows are asked for before anything else: the wait for tensor memory below overlaps their flight
+        if (FUSED) request_k_rows(0, n - n_late, 0, barK);
     }
     if (FUSED && warp == 1) fill_sector_table(sect, lane);
     // (the large size claims half of the SM's columns: two of the three resident CTAs hold theirs at a time, the
@@ -188,17 +200,22 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     if (BIG && (G || !similarity) && warp == 0) tmem_relinquish();  // this event takes no tensor memory
     if (BIG && !(G || !similarity) && warp == 0) tmem_alloc(smem_u32(tmem_holder), Cfg::kCols);
     tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
     const bool have_tmem = BIG ? (similarity && !G) : use_tc;
-    const uint32_t tbase = have_tmem ? *tmem_holder : 0u;
+    // The address of the columns is read after the next block-wide barrier: in the fused kernel that is the one
+    // that follows the position and statistic loads, so that warps 1..3 do those while warp 0 may still be
+    // waiting for columns.
+    uint32_t tbase = 0u;
+    if (!FUSED) {
+        __syncthreads();
+        tc_fence_after();
+        tbase = have_tmem ? *tmem_holder : 0u;
+    }
 
     phase_stamp(id.e, 1);
     // ---- scores ---------------------------------------------------------------------------------
     int bad = 0;
     int timeout = 0;
     if (FUSED) {
-        if (tid == 0) request_k_rows(0, n - n_late, 0, barK);
         const int* gpos = event_pos(a.pos, id);
         const bool rotate = gpos != nullptr;
         int pmax = INT_MIN;
@@ -218,6 +235,8 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             if (lane == 0) redi[warp] = pmax;
         }
         __syncthreads();
+        tc_fence_after();
+        tbase = have_tmem ? *tmem_holder : 0u;
         long long pref = 0;
         if (rotate) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)max(max(redi[0], redi[1]), max(redi[2], redi[3])) + 1;
         // lane covers frequencies f0..f0+7 of the row handled by its group of eight lanes
@@ -764,7 +783,9 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             *reinterpret_cast<uint4*>(Vg + off) = *reinterpret_cast<const uint4*>(src + 16384);
         }
     } else if ((unsigned)picks * 512u <= Cfg::kTileBytes) {
-        // the tile holds the kept rows of K and of V side by side: one round of loads, one barrier, one of stores
+        // The tile holds the kept rows of K and of V side by side: one round of 16-byte gathers, one barrier.
+        // Stores: slots 0..picks-1 are contiguous in a dense cache (and page by page in a paged one), so one
+        // thread writes them back with a few bulk copies. (Gathering by one bulk copy per row measured slower.)
         const uint32_t vhalf = Cfg::kTileBytes / 2u;
         for (int x = tid; x < picks * 16; x += kTcThreads) {
             const long long off = rowoff(idx[x >> 4]) + (x & 15) * 8;
@@ -772,11 +793,26 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
             cp_async16(tile_u32 + vhalf + (uint32_t)x * 16u, Vg + off);
         }
         cp_async_wait_all();
-        __syncthreads();
-        for (int x = tid; x < picks * 16; x += kTcThreads) {
-            const long long off = rowoff(x >> 4) + (x & 15) * 8;
-            copy16(reinterpret_cast<char*>(Kg + off), tile + x * 16);
-            copy16(reinterpret_cast<char*>(Vg + off), tile + vhalf + x * 16);
+        fence_proxy_async();  // the bulk stores below read what these copies wrote
+        __syncthreads();      // every kept row is on chip before the first store
+        const bool runs = dense ? lay.sn == kTcD : lay.s_page_n == kTcD;
+        if (runs) {
+            if (tid == 0) {
+                for (int row = 0; row < picks;) {
+                    const int run = dense ? picks - row : min(picks - row, lay.page_size - row % lay.page_size);
+                    const long long off = rowoff(row);
+                    bulk_s2g(Kg + off, tile_u32 + (uint32_t)row * 256u, (uint32_t)run * 256u);
+                    bulk_s2g(Vg + off, tile_u32 + vhalf + (uint32_t)row * 256u, (uint32_t)run * 256u);
+                    row += run;
+                }
+                bulk_store_wait_read();  // shared memory is read out before the CTA may leave
+            }
+        } else {
+            for (int x = tid; x < picks * 16; x += kTcThreads) {
+                const long long off = rowoff(x >> 4) + (x & 15) * 8;
+                copy16(reinterpret_cast<char*>(Kg + off), tile + x * 16);
+                copy16(reinterpret_cast<char*>(Vg + off), tile + vhalf + x * 16);
+            }
         }
     } else {
 #pragma unroll 1

@@ -131,7 +131,8 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     const uint32_t barM = bar_full + 128;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sp.misc + 136);
     int* cnt = reinterpret_cast<int*>(smem + sp.misc + 144);  // [0] a wait ran out, [1] newest position
-    const int nst = sp.stages;
+    const int nst = sp.stages;              // 8 or 4
+    const int nsh = nst == 8 ? 3 : 2;       // its logarithm: stage index and round of the ring by mask and shift
     const uint32_t tile_u32 = smem_u32(tile);
     const int cap = sp.cap_rows;
     const uint32_t half_bytes = (uint32_t)(cap + kStSpare) * 128u;
@@ -193,8 +194,8 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
     if (!worker) {
         if (lane == 0) {
             for (int st = 0; st < stages; ++st) {
-                const int sl = st % nst;
-                if (st >= nst && !mbar_wait_bounded(bar_empty + 8 * sl, (uint32_t)((st / nst - 1) & 1), a.wait_polls)) {
+                const int sl = st & (nst - 1);
+                if (st >= nst && !mbar_wait_bounded(bar_empty + 8 * sl, (uint32_t)(((st >> nsh) - 1) & 1), a.wait_polls)) {
                     atomicExch(&cnt[0], 1);
                     break;
                 }
@@ -220,9 +221,13 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
         const bool d_fits = (long long)D32 == D;
         ChainScore ca, cb;  // cb uses ca's S
         ca.set_step(D, phitab + f0, sect);
+        AKV_PHASE_ACC_DECL(cyc_kwait);
         for (int st = 0; st < stages; ++st) {
-            const int sl = st % nst;
-            if (!mbar_wait_bounded(bar_full + 8 * sl, (uint32_t)((st / nst) & 1), a.wait_polls)) {
+            const int sl = st & (nst - 1);
+            AKV_PHASE_ACC_BEGIN(cyc_kwait);
+            const bool landed = mbar_wait_bounded(bar_full + 8 * sl, (uint32_t)((st >> nsh) & 1), a.wait_polls);
+            AKV_PHASE_ACC_END(cyc_kwait);
+            if (!landed) {
                 atomicExch(&cnt[0], 1);
                 break;
             }
@@ -269,6 +274,7 @@ __global__ void __launch_bounds__(kStThreads, 1) event_stream_kernel(const Event
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_empty + 8 * sl) : "memory");
         }
+        AKV_PHASE_ACC_STORE(id.e, 13, cyc_kwait);
     }
     __syncthreads();
     if (cnt[0]) {

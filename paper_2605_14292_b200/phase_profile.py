@@ -82,6 +82,8 @@ def main():
     if kernel == "event_stream_kernel" and np.any(st[:, 10] > 0):
         for k, name in ((10, "  of picks: arg-max + exchange"), (11, "  of picks: products (misses)"), (12, "  of picks: tensor-memory read")):
             print(f"  {name:32s} {np.median(st[:, k]):10.0f} {st[:, k].mean():10.0f}")
+    if kernel == "event_stream_kernel" and np.any(st[:, 13] > 0):
+        print(f"  {'  of K streamed: warp 0 waiting for a stage':32s} {np.median(st[:, 13]):10.0f} {st[:, 13].mean():10.0f}")
     if kernel == "event_pool_kernel" and np.any(st[:, 10] > 0):
         ok = (st[:, 10] > 0) & (st[:, 1] > 0)
         d = (st[ok, 10] - st[ok, 1]).astype(np.float64)

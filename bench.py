@@ -53,6 +53,16 @@ KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_pool_kernel<fused>
 # keyed by workload, each with the source revision of csrc/ it was taken at (see kernel_revision()); a
 # capture of another revision is reported as null.
 NCU_TRAFFIC = {
+    # one launch of 4096 events captured whole (profiles/event_tri_kernel_bf16_C3.md)
+    "C3": {"bytes": 323942144 + 99312128, "revision": "46fd6f6dbfe6"},
+    # one launch of 4096 events (16 sequences) captured; a step is 4 x 32 launches of that size
+    # (profiles/event_pool_kernel_bf16_C5.md)
+    "C5": {"bytes": (490665984 + 230640384) * 128, "revision": "46fd6f6dbfe6"},
+    # the same kernel and capture, scaled to 112 events
+    "C2": {"bytes": (490665984 + 230640384) * 112 // 4096, "revision": "46fd6f6dbfe6"},
+    # the three launches (lambda 0, 0.5, 1) of a 2-sequence batch captured; the bench batch has 8 sequences
+    # (profiles/event_stream_kernel_bf16_C4.md)
+    "C4": {"bytes": ((249031424 + 12117760) + (256561152 + 10830080) + (256438784 + 10525440)) * 4, "revision": "46fd6f6dbfe6"},
 }
 
 
@@ -174,19 +184,26 @@ def oracle_sample(config: str, seed: int = 0):
     return ev, [0.5], "512 of 16384 events (batch 2 of 64), the first of the 32 events only", 1
 
 
-def oracle_time(ev, lams, reps=1, threads=None):
-    """Times the C oracle, as it stands, on whole events of `ev` with `threads` host threads."""
+def oracle_time(ev, lams, reps=1, threads=None, min_seconds=0.0):
+    """Times the C oracle, as it stands, on whole events of `ev` with `threads` host threads: `reps` passes
+    over the sample, repeated until `min_seconds` of wall time have gone by. Returns events/s, threads, seconds
+    and the events processed."""
     from oracle import c_oracle as CO
     threads = threads or (os.cpu_count() or 1)
     CO.build()
     E = ev.n_events
     CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lams[0], events=(0, min(E, threads)), threads=threads)
+    done = 0
     t0 = time.perf_counter()
-    for _ in range(reps):
-        for lam in lams:
-            CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lam, threads=threads)
-    dt = time.perf_counter() - t0
-    return E * reps * len(lams) / dt, threads, dt
+    while True:
+        for _ in range(reps):
+            for lam in lams:
+                CO.event_batch(ev.K, ev.V, ev.pos, ev.qstat, ev.p_ref, ev.budget, lam, threads=threads)
+        done += E * reps * len(lams)
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds:
+            break
+    return done / dt, threads, dt, done
 
 
 def flat_oracle_time(ev, lams):
@@ -212,17 +229,17 @@ def cpu_baseline(config: str):
         return {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "sample": f"{what}, NumPy oracle in float64, {dt:.1f} s wall in one process",
                 "single_thread": {"value": v, "events": ev.n_events, "wall_s": round(dt, 2)}}
-    v, threads, dt = oracle_time(ev, lams, reps)
+    v, threads, dt, done = oracle_time(ev, lams, reps, min_seconds=10.0)
     # one thread on a smaller slice of the same sample
     one = ev
     if ev.n_events > 32:
         from paper_2605_14292_b200 import synth
         one = synth.EventBatch(ev.name, ev.dtype, ev.K[:1, :2], ev.V[:1, :2], ev.pos[:1, :2], ev.qstat[:2], ev.p_ref[:1],
                                ev.budget, ev.lam)
-    v1, _, dt1 = oracle_time(one, lams, reps, threads=1)
+    v1, _, dt1, done1 = oracle_time(one, lams, reps, threads=1, min_seconds=5.0)
     return {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{what}, C oracle in float64, {dt:.1f} s wall on {threads} threads",
-            "single_thread": {"value": v1, "events": one.n_events * len(lams) * reps, "wall_s": round(dt1, 2)}}
+            "sample": f"{what}, repeated to {done} events, C oracle in float64, {dt:.1f} s wall on {threads} threads",
+            "single_thread": {"value": v1, "events": done1, "wall_s": round(dt1, 2)}}
 
 
 def run_reference(args):
@@ -231,17 +248,25 @@ def run_reference(args):
         return
     ev, lams, what, reps = oracle_sample(args.config)
     threads = os.cpu_count() or 1
-    run = (lambda: flat_oracle_time(ev, lams)) if args.config == "C6" else (lambda: oracle_time(ev, lams, reps, threads))
+    # a step repeats the sample for about a second (less when many steps are asked for: the whole run stays
+    # within two minutes or so)
+    per_step = min(1.0, 100.0 / max(args.steps + args.warmup, 1))
     if args.config == "C6":
         threads = 1
+        work = lambda: flat_oracle_time(ev, lams)
+    else:
+        work = lambda: oracle_time(ev, lams, reps, threads, min_seconds=per_step)
+    events = 0
     for _ in range(args.warmup):
-        run()
+        work()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        run()
+        r = work()
+        events += r[3] if len(r) > 3 else ev.n_events * len(lams)
     dt = time.perf_counter() - t0
-    value = ev.n_events * len(lams) * reps * args.steps / dt
-    sample = f"per step: {what}, {'NumPy' if args.config == 'C6' else 'C'} oracle in float64, {threads} threads"
+    value = events / dt
+    sample = (f"per step: {what}, repeated for {per_step:.2f} s, {'NumPy' if args.config == 'C6' else 'C'} oracle in float64, "
+              f"{threads} threads")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",

@@ -7,8 +7,9 @@
 //   therefore formed only for the pool's best-scored rows, at most 180 of them (64 KB of triangle: three CTAs
 //   per SM), and only their V rows are read. Every candidate left out scores at most `bound`, the 181st largest
 //   key, and its Eq. 2 value never exceeds its score: the loop over the active set is exact as long as its
-//   winning value stays above that bound. In the rare event where it does not, the event is redone over its whole
-//   pool with rows of the cosine matrix taken as plain dot products.
+//   winning value stays above that bound. In the rare event where it does not, the picks made so far stand and
+//   the remaining ones (a few, as a rule) are taken over the whole pool with rows of the cosine matrix as plain
+//   dot products, starting from the running maxima the loop had reached.
 //
 //   Rows 128.. of the active set: a second product (the operand's last 128 rows against rows 128..) gives their
 //   cosines against one another; their cosines against rows < 128 are those rows' columns 128.. by symmetry.
@@ -20,6 +21,11 @@ namespace akv {
 // Two sizes of the kernel. The small one (budgets up to 64): a tile of 128 rows of 256 bytes, which holds the V
 // operand and then the triangle of a pool of up to 127 rows; six CTAs per SM. The large one (budgets up to 128,
 // N up to 256): 64 KB, for a whole event's K rows, then the triangle of an active set of up to 180 rows (see the kernel); three CTAs per SM.
+// Scratch of the continuation after the active set's bound was reached, as byte offsets into the tile (the triangle
+// is dead by then): the loop's running maxima, and behind the plain-dot route's row buffer the arrays of the hand-over.
+constexpr unsigned kContScratch = 2048u;   // 2 KB + 2 x 1 KB + 2 x 512 B + 512 B + 256 B + 4 B
+constexpr unsigned kContMact = 8192u;      // 1 KB
+
 template <bool BIG>
 struct TriCfg {
     static constexpr unsigned kTileBytes = BIG ? 65536u : 32768u;
@@ -265,7 +271,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                 // G follows from the previous round's by the constant turn when all four rows of the warp sit
                 // D16 after the rows 16 slots before them
                 bool fresh = (round & (kChainRoundsShort - 1)) == 0 || a.no_chain;
-                if (!fresh) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - 16] == D16);
+                if (!fresh && !uniform) fresh = !__all_sync(0xFFFFFFFFu, !live || (long long)spos[j] - (long long)spos[j - 16] == D16);
                 if (fresh) {
                     if (live) cs.anchor(pref - (long long)spos[j], gtab + f0, phitab + f0, sect);
                 } else {
@@ -471,6 +477,7 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     const uint32_t bound_key = BIG ? *bound_holder : 0u;
     const bool fast = similarity && P <= Cfg::kMaxPool && picks > 1;
     bool slow = similarity && P > Cfg::kMaxPool;  // (small size only; the large size may set it after its loop)
+    int cont_from = -1;                           // large size: picks already made when the bound was reached
 
     phase_stamp(id.e, 3);
     // ---- V rows of the pool as the swizzled operand tile ---------------------------------------------
@@ -646,7 +653,8 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
     if (!slow) {
         if (warp == 0) {
             if (BIG) {
-                const bool ok = fast ? picks_cosine<Cfg::kCpl, true>(lane, P, picks, s, bypool, r, a.lam, tri, park_key, order, bound_key)
+                const bool ok = fast ? picks_cosine<Cfg::kCpl, true>(lane, P, picks, s, bypool, r, a.lam, tri, park_key, order, bound_key,
+                                                                     reinterpret_cast<float*>(tile + kContMact), redi)
                                      : picks_bounded<8>(lane, P, picks, false, s, bypool, r, a.lam, tri, park_key, order);
                 if (lane == 0) *pick_holder = ok ? 0 : -2;
             } else if (P <= 128) {
@@ -658,9 +666,31 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
         if (BIG) {
             __syncthreads();
             if (*pick_holder == -2) {
-                // a winning value fell to the bound: the event is redone over its whole pool, rows of the cosine
-                // matrix by plain dot products (below)
+                // A winning value fell to the bound with `done` picks made. Those stand (no left-out candidate could
+                // have won them). The rest of the picks, a few as a rule, are taken over the whole pool with rows of
+                // the cosine matrix as plain dot products (below), from the state the loop left: its running maxima
+                // for the rows it had, and for the rows it had left out the maximum over the picks made, formed here.
                 slow = true;
+                cont_from = redi[0];
+                const int done = cont_from;
+                float* m_act = reinterpret_cast<float*>(tile + kContMact);                  // by old pool row (from the loop)
+                float* m_slot = reinterpret_cast<float*>(tile + kContScratch);              // by slot
+                float* m_init = m_slot + 256;                                               // by new pool row
+                unsigned short* inv = reinterpret_cast<unsigned short*>(m_init + 256);      // slot -> new pool row
+                unsigned short* left = inv + 256;                                           // new pool rows the loop had left out
+                int* chosen = reinterpret_cast<int*>(left + 256);                           // slots of the picks made
+                unsigned char* state = reinterpret_cast<unsigned char*>(chosen + 128);      // by slot: 1 in the old active set
+                int* n_left = reinterpret_cast<int*>(state + 256);
+                for (int j = tid; j < 256; j += kTcThreads) state[j] = 0;
+                if (tid == 0) *n_left = 0;
+                __syncthreads();
+                for (int rho = tid; rho < P; rho += kTcThreads) {
+                    const int j = bypool[rho];
+                    state[j] = 1;
+                    m_slot[j] = m_act[rho];
+                }
+                for (int t = tid; t < done; t += kTcThreads) chosen[t] = bypool[order[t]];
+                __syncthreads();
                 if (warp == 0) {
                     const float thr = *thr_holder;
                     int base = 0;
@@ -677,8 +707,16 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                 __syncthreads();
                 P = *pool_holder;
                 for (int rho = tid; rho < P; rho += kTcThreads) {
+                    const int j = bypool[rho];
+                    inv[j] = (unsigned short)rho;
+                    if (state[j]) {
+                        m_init[rho] = m_slot[j];
+                    } else {
+                        m_init[rho] = 0.f;
+                        left[atomicAdd(n_left, 1)] = (unsigned short)rho;
+                    }
                     if (G) { r[rho] = 1.f; continue; }
-                    const __nv_bfloat16* vrow = Vg + rowoff(bypool[rho]);
+                    const __nv_bfloat16* vrow = Vg + rowoff(j);
                     float ss = 0.f;
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
@@ -690,13 +728,56 @@ __global__ void __launch_bounds__(kTcThreads, BIG ? 3 : 7) event_pool_kernel(con
                     r[rho] = 1.f / (sqrtf(ss) + a.eps);
                 }
                 __syncthreads();
+                for (int t = tid; t < done; t += kTcThreads) order[t] = inv[chosen[t]];
+                __syncthreads();
+                // left-out rows against the picks made: m = max(0, max_t r_t <V_c, V_t>), every (row, pick) pair its own
+                // dot product, the maximum by an integer atomic (the values are non-negative floats)
+                const int pairs = *n_left * done;
+                for (int x = tid; x < pairs; x += kTcThreads) {
+                    const int c = left[x / done], i = order[x % done];
+                    float acc;
+                    if (G) {
+                        acc = G[(long long)bypool[i] * N + bypool[c]];
+                    } else {
+                        const __nv_bfloat16* vi = Vg + rowoff(bypool[i]);
+                        const __nv_bfloat16* vc = Vg + rowoff(bypool[c]);
+                        acc = 0.f;
+#pragma unroll 4
+                        for (int q = 0; q < 16; ++q) {
+                            float xi[8], xc[8];
+                            load8(vi + q * 8, xi);
+                            load8(vc + q * 8, xc);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc = fmaf(xi[e], xc[e], acc);
+                        }
+                    }
+                    const float v = fmaxf(r[i] * acc, 0.f);
+                    atomicMax(reinterpret_cast<int*>(m_init) + c, __float_as_int(v));
+                }
+                __syncthreads();
             }
         }
     }
     if (slow) {
         GreedyLane<8> g;
-        if (warp == 0) g.init(lane, P, s, bypool, r, a.lam, true);
-        for (int t = 0; t < picks; ++t) {
+        if (warp == 0) {
+            g.init(lane, P, s, bypool, r, a.lam, true);
+            if (BIG && cont_from >= 0) {
+                // continue after the picks the bounded loop made: its maxima, and those picks out of the running
+                // (rowbuf, the first 1 KB of the tile, is written by the loop below; the scratch lies behind it)
+                const float* m_init = reinterpret_cast<const float*>(tile + kContScratch) + 256;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int rho = lane + 32 * k;
+                    if (rho < P) {
+                        const float m0 = m_init[rho];
+                        g.M[k] = m0;
+                        if (m0 == __int_as_float(0x7f800000)) g.am[k] = 0u;  // picked already (the loop's +inf)
+                    }
+                }
+            }
+        }
+        for (int t = BIG && cont_from > 0 ? cont_from : 0; t < picks; ++t) {
             if (warp == 0) {
                 uint32_t bk;
                 const int irho = g.pick(lane, bk);

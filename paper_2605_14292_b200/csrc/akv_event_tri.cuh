@@ -193,11 +193,12 @@ constexpr float kLowestScore = -3.0e38f;
 // pick, so the update m <- max(m, Sims[i, :]) gives the picked row m = +inf and a = -inf from then on: no
 // mask, no per-candidate retirement. Each lane reduces its candidates to one maximum before the warp-wide
 // reduction and finds which candidate that was while the reduction is in flight. Winning values are parked as order-preserving keys, like the other loops'.
-// BOUNDED as for picks_bounded. `tri` is modified (its diagonal).
+// BOUNDED as for picks_bounded; when the bound is reached the state of the loop can be handed back (see there).
+// `tri` is modified (its diagonal).
 template <int CPL, bool BOUNDED>
 __device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const float* s, const unsigned short* bypool,
                                              const float* r, float lam, float* tri, uint32_t* park_key, int* park_row,
-                                             uint32_t bound_key = 0u) {
+                                             uint32_t bound_key = 0u, float* m_out = nullptr, int* t_out = nullptr) {
     const uint32_t tb = smem_u32(tri), rb = smem_u32(r);
     const float ninf = __int_as_float(0xff800000), pinf = __int_as_float(0x7f800000);
     float sv[CPL], lr[CPL], M[CPL];
@@ -248,7 +249,22 @@ __device__ __forceinline__ bool picks_cosine(int lane, int P, int picks, const f
             const int row = bi[0];
             const uint32_t wlo = __reduce_max_sync(0xFFFFFFFFu, lm == whi ? 0xFFFFu - (uint32_t)row : 0u);
             const int irho = min((int)(0xFFFFu - wlo), last);
-            if (BOUNDED && whi <= bound) return false;
+            if (BOUNDED && whi <= bound) {
+                // The picks made so far stand. They are parked, and with m_out / t_out given the running maxima
+                // (by pool row; +inf for the rows already picked) and the number of picks are left for the caller
+                // to continue from.
+                if (t0 + lane < t) {
+                    park_key[t0 + lane] = orderable(my_val <= -2.9e38f ? ninf : my_val);
+                    park_row[t0 + lane] = my_row;
+                }
+                if (m_out) {
+#pragma unroll
+                    for (int k = 0; k < CPL; ++k)
+                        if (lane + 32 * k < P) m_out[lane + 32 * k] = M[k];
+                }
+                if (t_out && lane == 0) *t_out = t;
+                return false;
+            }
             const bool mine = lane == t - t0;
             my_val = mine ? whi : my_val;
             my_row = mine ? irho : my_row;

@@ -559,6 +559,48 @@ def test_fused_event_with_shared_cosine_matrix(mode, N, budget):
     assert int(sel.status.abs().max()) == 0 and int(sel.n_kept.min()) == budget
 
 
+def _duplicated_rows(seed, lam, B=2, L=2, H=2, N=256, budget=128):
+    """Every V row occurs twice (rows j and j + N/2 are bit-identical): once a row is picked its twin is
+    penalised by lambda, so the picks must go far down the score order, beyond any active set."""
+    ev = synth.make_plain(B, L, H, N, 128, budget, lam, dtype=synth.BF16, seed=seed)
+    ev.V[..., N // 2:, :] = ev.V[..., :N // 2, :]
+    return ev
+
+
+@pytest.mark.parametrize("lam", [2.0, 1.5])
+def test_active_set_bound_reached_and_the_loop_continues_over_the_whole_pool(lam):
+    """N = 256 -> b = 128 with duplicated V rows: the one-warp loop over the best-scored rows reaches its bound;
+    the picks made stand, the rest are taken over the whole pool. Every pick is checked against the oracle."""
+    ev = _duplicated_rows(33, lam)
+    g = run_fused(ev, lam=lam)
+    log = check_all(ev, g, lam)
+    # the picks did go deep: some kept row's score rank lies beyond the 180 rows an active set holds at most
+    s = g["scores"][0, 0, 0]
+    rank = np.argsort(np.argsort(-s))
+    assert rank[g["idx"][0, 0, 0]].max() >= 181
+    print("duplicated rows, lambda", lam, "near-tie divergences:", log)
+
+
+def test_active_set_bound_reached_with_a_shared_cosine_matrix():
+    """The same with Eq. 1 signatures and one cosine matrix per sequence (one layer, one head: the flat signature
+    is the head's own), so the continuation reads its cosines from that matrix."""
+    lam = 1.5
+    ev = _duplicated_rows(34, lam, B=2, L=1, H=1)
+    K, V, pos, q, pref = dev(ev.K), dev(ev.V), dev(ev.pos), dev(ev.qstat), dev(ev.p_ref)
+    sig = akv.alpha_signature_flat(V)
+    gram = akv.alpha_gram_shared(sig, akv.Layout.dense(V), akv.Options(sig_mode=akv.SIG_FLAT))
+    sel = akv.alpha_compress_event(K, V, pos, q, ev.budget, akv.Options(lam=lam, sig_mode=akv.SIG_FLAT, shared_gram=gram),
+                                   p_ref=pref, flat_sig=sig, want_scores=True)
+    torch.cuda.synchronize()
+    Kn, Vn, pn = akv.to_host_bits(K), akv.to_host_bits(V), pos.cpu().numpy()
+    for b in range(2):
+        chk.check_event(ev.K[b, 0, 0], ev.V[b, 0, 0], ev.pos[b, 0, 0], ev.qstat[0, 0], int(ev.p_ref[b]), ev.budget, lam,
+                        sel.scores[b, 0, 0].cpu().numpy(), sel.pick_order[b, 0, 0].cpu().numpy(),
+                        sel.idx_sorted[b, 0, 0].cpu().numpy(), Kn[b, 0, 0], Vn[b, 0, 0], pn[b, 0, 0],
+                        sig=O.signatures_flat(ev.V[b]))
+    assert int(sel.status.abs().max()) == 0 and int(sel.n_kept.min()) == ev.budget
+
+
 # ------------------------------------------------------------------ grouped-query statistics
 @pytest.mark.parametrize("reduce", ["mean", "max"])
 @pytest.mark.parametrize("dtype,N,d", [(synth.BF16, 150, 128), (synth.F32, 600, 64)])

@@ -132,125 +132,6 @@ __host__ __device__ inline SmemPlan plan_smem(int N, int d, int esize, int budge
     return p;
 }
 
-// copy n rows of one event between global memory and a dense shared tile, 16 bytes per thread and step
-template <typename T>
-__device__ __forceinline__ void load_tile(T* tile, const T* base, const DevLayout& lay, const EventId& id, int n) {
-    const int cpr = lay.d * (int)sizeof(T) / 16;  // 16-byte chunks per row
-    for (int x = threadIdx.x; x < n * cpr; x += kThreads) {
-        const int row = x / cpr, c = x - row * cpr;
-        const char* src = reinterpret_cast<const char*>(base + row_offset(lay, id.b, id.l, id.h, row)) + c * 16;
-        copy16(reinterpret_cast<char*>(tile) + (size_t)x * 16, src);
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Fused event, tiles resident in shared memory: K and V are read from HBM once and the kept rows
-// are written once. One CTA per (sequence, layer, KV head).
-// ---------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(kThreads) event_resident_kernel(const EventArgs a, const __grid_constant__ ScoreTab tab) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    const DevLayout& lay = a.lay;
-    const EventId id = decode_event(lay, blockIdx.x);
-    const int n = event_n(a, id.b);
-    const int d = lay.d, N = lay.N;
-    const SmemPlan sp = plan_smem(N, d, sizeof(T), a.budget, true, true);
-    T* Kt = reinterpret_cast<T*>(smem + sp.tileK);
-    T* Vt = reinterpret_cast<T*>(smem + sp.tileV);
-    unsigned long long* phi = reinterpret_cast<unsigned long long*>(smem + sp.phi);
-    float2* g = reinterpret_cast<float2*>(smem + sp.g);
-    int* spos = reinterpret_cast<int*>(smem + sp.pos);
-    float* s = reinterpret_cast<float*>(smem + sp.s);
-    float* r = reinterpret_cast<float*>(smem + sp.r);
-    float* m = reinterpret_cast<float*>(smem + sp.m);
-    int* order = reinterpret_cast<int*>(smem + sp.order);
-    float* gain = reinterpret_cast<float*>(smem + sp.gain);
-    int* idx = reinterpret_cast<int*>(smem + sp.idx);
-    unsigned char* taken = smem + sp.taken;
-    unsigned long long* red = reinterpret_cast<unsigned long long*>(smem + sp.red);
-    int* redi = reinterpret_cast<int*>(smem + sp.red + 2 * kWarps * 8);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int* gpos = event_pos(a.pos, id);
-    T* Kg = reinterpret_cast<T*>(a.K);
-    T* Vg = reinterpret_cast<T*>(a.V);
-
-    // stage the event on chip
-    load_tile(Kt, Kg, lay, id, n);
-    load_tile(Vt, Vg, lay, id, n);
-    int pmax = INT_MIN;
-    for (int j = tid; j < n; j += kThreads) {
-        const int p = gpos ? gpos[j] : 0;
-        spos[j] = p;
-        pmax = max(pmax, p);
-        taken[j] = 0;
-        m[j] = 0.f;
-    }
-    for (int f = tid; f < d / 2; f += kThreads) phi[f] = tab.phi[f];
-    const int members = fold_group(a, id, tab, d, g);
-    long long pref = 0;
-    if (gpos) pref = a.p_ref ? (long long)a.p_ref[id.b] : (long long)block_max_int(pmax, redi) + 1;
-    __syncthreads();
-
-    // scores and reciprocal norms
-    const int G = pow2_ceil(d >> 3) > 32 ? 32 : pow2_ceil(d >> 3);
-    const int RPW = 32 / G, grp = lane / G, lig = lane % G;
-    int bad = 0;
-    for (int j0 = warp * RPW; j0 < n; j0 += kWarps * RPW) {
-        const int j = j0 + grp;
-        const bool valid = j < n;
-        const long long dist = valid ? pref - (long long)spos[j] : 0;
-        const float sc = score_group(Kt + (size_t)j * d, valid, dist, gpos != nullptr, d, phi, g, lig, G, members);
-        const float ss = a.flat_sig ? 1.f : sumsq_row(Vt + (size_t)j * d, valid, d, lig, G);
-        if (valid && lig == 0) {
-            if (a.scores) a.scores[(long long)id.e * N + j] = sc;
-            const bool fin = isfinite(sc);
-            bad |= !fin;
-            s[j] = fin ? sc : -INFINITY;
-            r[j] = 1.f / (sqrtf(ss) + a.eps);
-        }
-    }
-    bad = __syncthreads_or(bad);
-
-    // selection
-    const int bud = event_budget(a, id);
-    const int picks = min(bud, n);
-    if (a.flat_sig) {
-        StridedRows<float> rows{event_sig(a, id), d};
-        greedy_cta<float>(n, picks, a.lam, a.greedy != 0, d, s, nullptr, m, taken, order, gain, rows, red);
-    } else {
-        StridedRows<T> rows{Vt, d};
-        greedy_cta<T>(n, picks, a.lam, a.greedy != 0, d, s, r, m, taken, order, gain, rows, red);
-    }
-    ordered_indices(n, a.budget, taken, idx);
-    __syncthreads();
-
-    // outputs
-    const long long ob = (long long)id.e * a.budget;
-    for (int t = tid; t < a.budget; t += kThreads) {
-        a.idx_sorted[ob + t] = idx[t];
-        if (a.pick_order) a.pick_order[ob + t] = t < picks ? order[t] : -1;
-        if (a.pick_gain) a.pick_gain[ob + t] = t < picks ? gain[t] : 0.f;
-    }
-    if (tid == 0) {
-        if (a.n_kept) a.n_kept[id.e] = picks;
-        if (a.status) a.status[id.e] = n < bud ? 2 : (bad ? 1 : 0);
-    }
-    // compaction: kept rows go to slots 0..picks-1 of the same buffer (all sources are on chip)
-    const int cpr = d * (int)sizeof(T) / 16;
-    for (int x = tid; x < picks * cpr; x += kThreads) {
-        const int rr = x / cpr, c = x - rr * cpr;
-        const int src = idx[rr];
-        const long long off = row_offset(lay, id.b, id.l, id.h, rr);
-        copy16(reinterpret_cast<char*>(Kg + off) + c * 16, reinterpret_cast<const char*>(Kt + (size_t)src * d) + c * 16);
-        copy16(reinterpret_cast<char*>(Vg + off) + c * 16, reinterpret_cast<const char*>(Vt + (size_t)src * d) + c * 16);
-    }
-    if (gpos) {
-        int* wpos = a.pos.p + id.b * a.pos.sb + id.l * a.pos.sl + id.h * a.pos.sh;
-        for (int t = tid; t < picks; t += kThreads) wpos[t] = spos[idx[t]];
-    }
-}
-
 // ---------------------------------------------------------------------------------------------
 // Stand-alone score: one CTA per (event, block of kScoreRows rows), both folded into grid.x; K
 // streamed from global memory once.

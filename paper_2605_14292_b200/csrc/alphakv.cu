@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstring>
 
+#include "akv_event_general.cuh"
 #include "akv_event_pool.cuh"
 #include "akv_event_stream.cuh"
 #include "akv_gram.cuh"
@@ -613,12 +614,19 @@ static akv_status_t alpha_compress_event_impl(akv_handle_t* h, const akv_layout_
         const int es = lay->dtype == AKV_BF16 ? 2 : 4;
         const SmemPlan res = plan_smem(lay->N, lay->d, es, budget, true, true);
         const int E = a.lay.B * a.lay.L * a.lay.H;
+        // beside the tiles: the pool's list and norms and as much of a cosine triangle as the SM's shared memory
+        // leaves room for (at most the whole event's)
+        const long long whole = (long long)align16((unsigned)lay->N * 2u) + align16((unsigned)lay->N * 4u) +
+                                (long long)lay->N * (lay->N + 1) / 2 * 4;
+        const long long room = (long long)h->smem_optin - (long long)res.total;
+        const int extra = (int)((room < whole ? room : whole) & ~15ll);
+        const unsigned total = res.total + (unsigned)(extra > 0 ? extra : 0);
         if (lay->dtype == AKV_BF16) {
-            if ((s = set_smem(event_resident_kernel<__nv_bfloat16>, res.total)) != AKV_OK) return s;
-            event_resident_kernel<__nv_bfloat16><<<E, kThreads, res.total, st>>>(a, h->tab);
+            if ((s = set_smem(event_resident_kernel<__nv_bfloat16>, total)) != AKV_OK) return s;
+            event_resident_kernel<__nv_bfloat16><<<E, kThreads, total, st>>>(a, h->tab, extra > 0 ? extra : 0);
         } else {
-            if ((s = set_smem(event_resident_kernel<float>, res.total)) != AKV_OK) return s;
-            event_resident_kernel<float><<<E, kThreads, res.total, st>>>(a, h->tab);
+            if ((s = set_smem(event_resident_kernel<float>, total)) != AKV_OK) return s;
+            event_resident_kernel<float><<<E, kThreads, total, st>>>(a, h->tab, extra > 0 ? extra : 0);
         }
         return launched("event");
     }

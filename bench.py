@@ -54,15 +54,15 @@ KERNELS = {"C1": "event_resident_kernel<float>", "C2": "event_pool_kernel<fused>
 # capture of another revision is reported as null.
 NCU_TRAFFIC = {
     # one launch of 4096 events captured whole (profiles/event_tri_kernel_bf16_C3.md)
-    "C3": {"bytes": 324261632 + 99401728, "revision": "5adb947c4c32"},
+    "C3": {"bytes": 323675904 + 98740992, "revision": "2ef03d00f108"},
     # one launch of 4096 events (16 sequences) captured; a step is 4 x 32 launches of that size
     # (profiles/event_pool_kernel_bf16_C5.md)
-    "C5": {"bytes": (489598720 + 229892608) * 128, "revision": "5adb947c4c32"},
+    "C5": {"bytes": (489861376 + 230915584) * 128, "revision": "2ef03d00f108"},
     # the same kernel and capture, scaled to 112 events
-    "C2": {"bytes": (489598720 + 229892608) * 112 // 4096, "revision": "5adb947c4c32"},
+    "C2": {"bytes": (489861376 + 230915584) * 112 // 4096, "revision": "2ef03d00f108"},
     # the three launches (lambda 0, 0.5, 1) of a 2-sequence batch captured; the bench batch has 8 sequences
     # (profiles/event_stream_kernel_bf16_C4.md)
-    "C4": {"bytes": ((249034240 + 11675648) + (256383744 + 11495936) + (256425216 + 11520256)) * 4, "revision": "5adb947c4c32"},
+    "C4": {"bytes": ((249109504 + 12716032) + (256418560 + 10868480) + (256417536 + 11575296)) * 4, "revision": "2ef03d00f108"},
 }
 
 
